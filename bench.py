@@ -1,0 +1,346 @@
+#!/usr/bin/env python
+"""Benchmark of the sparse MLA decode path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One step = one call of omni_sparse_mla_decode (main kernel + split-KV merge) over one batch of
+the DeepSeek-R1-shaped decode workload (batch 32, 128 heads, 32768-token contexts, 2112 selected
+tokens per request, shuffled 64-token pages).  Prints ONE JSON line on rank 0.
+
+Metric: selected-KV bandwidth = 1152 bytes x selected tokens / step time (GB/s), with the step
+time in microseconds beside it.  Requests are independent, so with N > 1 every rank runs its own
+batch (weak scaling, no collective on the data path) and the value is the sum over ranks divided
+by the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+KV_ROW_BYTES = 1152
+FLOP_PER_TOKEN_HEAD = 2 * (576 + 512)
+L2_BYTES = 126 * 1024 * 1024
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm=float(p["hbm_gbs"]), tc_burst=float(p["bf16_tflops"]),
+                    tc_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
+    return dict(hbm=6650.0, tc_burst=1590.0, tc_sustained=1400.0, source="fallback")
+
+
+def _kernel_source_hash():
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_2511_22481_b200", "csrc")
+    for name in sorted(os.listdir(csrc)):
+        with open(os.path.join(csrc, name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def _recorded_traffic(kernel_hash):
+    """DRAM bytes per launch of the dominant kernel from the committed ncu summary, or None if
+    there is none or the kernel sources changed since the counters were taken."""
+    path = os.path.join(ROOT, "profiles", "dominant_kernel_traffic.json")
+    if not os.path.exists(path):
+        return None
+    with open(path) as f:
+        rec = json.load(f)
+    if rec.get("kernel_source_hash") != kernel_hash:
+        return None
+    return rec.get("dram_bytes_per_launch")
+
+
+class ClockSampler:
+    """nvidia-smi polling in a child process while the timed region runs."""
+
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.QUERY,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return dict(sm_mhz=statistics.median(sm) if sm else None,
+                    sm_max_mhz=max(mx) if mx else None, samples=len(sm), reasons=sorted(reasons))
+
+
+def _oracle_sample(w, target_s=15.0, max_requests=None):
+    """Time the CPU oracle, as it stands, on the first requests of the workload (all heads)."""
+    import numpy as np
+    import torch
+    import oracle
+
+    def run(reqs):
+        pt = w.page_table[reqs].cpu().numpy()
+        si = w.sel_idx[reqs].cpu().numpy()
+        sl = w.sel_len[reqs].cpu().numpy()
+        rows = oracle.resolve_rows(pt, si, sl, w.page_size, w.num_pages)
+        gather = torch.from_numpy(np.where(rows < 0, 0, rows)).to(w.kv_cache.device)
+        krows = w.kv_cache.view(-1, w.d_qk)[gather.view(-1)].view(len(reqs), -1, w.d_qk).cpu()
+        q = w.q[reqs].cpu()
+        t0 = time.perf_counter()
+        oracle.attend_rows(q, krows, sl, w.d_v, w.scale)
+        return time.perf_counter() - t0, int(sl.sum())
+
+    t1, _ = run(slice(0, 1))
+    n = max(1, min(w.batch if max_requests is None else max_requests, int(target_s / max(t1, 1e-3))))
+    t, tokens = run(slice(0, n))
+    return dict(seconds=t, tokens=tokens, requests=n, cores=oracle.num_threads())
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--kernel", default="tc", choices=["tc", "simt"],
+                    help="tc: tensor-core kernel (the product path); simt: plain-FMA bring-up kernel")
+    ap.add_argument("--clones", type=int, default=6, help="KV pool copies rotated to keep L2 cold")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        if rank != 0:
+            return 0
+        return reference_arm(args)
+
+    import torch
+    import torch.distributed as dist
+    from paper_2511_22481_b200 import binding as B
+    from paper_2511_22481_b200 import build as builder
+    from paper_2511_22481_b200 import workloads as W
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+    builder.build()
+    B.load()
+
+    flags = B.OMNI_FLAG_SIMT if args.kernel == "simt" else 0
+    w = W.config2_r1(dev)
+    # keep L2 cold: rotate over independent copies of the pool so the bytes touched between two
+    # uses of the same copy exceed L2 several times
+    clones = max(2, args.clones)
+    pools = [w.kv_cache] + [w.kv_cache.clone() for _ in range(clones - 1)]
+    plan = B.plan_for(w, flags=flags)
+    kv_bytes = w.selected_kv_bytes
+    flops = w.selected_tokens * w.heads * FLOP_PER_TOKEN_HEAD
+    launches_per_step = 1 + (1 if plan.splits > 1 else 0)
+
+    def step(i, ev=None):
+        if ev is not None:
+            B.omni_sparse_mla_set_profile_events(ev[0], ev[1])
+        B.omni_sparse_mla_decode(plan.desc, w.q, pools[i % clones], w.page_table, w.sel_idx,
+                                 w.sel_len, plan.out, plan.lse, plan.workspace, plan.status)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing --------------------------------------------------------
+    kern_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+               for _ in range(args.steps)]
+    for a, b in kern_ev:                      # materialise the events before handing them to C
+        a.record()
+        b.record()
+    for i in range(args.warmup):
+        step(i)
+    sampler = ClockSampler(local_rank)
+    barrier()
+    sampler.start()
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_begin.record()
+    for i in range(args.steps):
+        step(args.warmup + i, kern_ev[i])
+    t_end.record()
+    barrier()
+    B.omni_sparse_mla_set_profile_events(None, None)
+    clocks = sampler.stop()
+    ms_total = t_begin.elapsed_time(t_end)
+    kern_ms = [a.elapsed_time(b) for a, b in kern_ev]
+    status = int(plan.status.item())
+    if status != 0:
+        raise SystemExit("device status word is %d after the timed region" % status)
+
+    # ---- end to end through the host-buffer entry point ---------------------------------
+    staging = torch.empty(B.omni_sparse_mla_host_staging_bytes(plan.desc), dtype=torch.uint8, device=dev)
+    q_h, pt_h = w.q.cpu().pin_memory(), w.page_table.cpu().pin_memory()
+    si_h, sl_h = w.sel_idx.cpu().pin_memory(), w.sel_len.cpu().pin_memory()
+    out_h = torch.empty(plan.out.shape, dtype=torch.bfloat16).pin_memory()
+    lse_h = torch.empty(plan.lse.shape, dtype=torch.float32).pin_memory()
+    h2d = sum(t.numel() * t.element_size() for t in (q_h, pt_h, si_h, sl_h))
+    d2h = sum(t.numel() * t.element_size() for t in (out_h, lse_h))
+
+    def e2e_step(i):
+        B.omni_sparse_mla_decode_host(plan.desc, q_h, pools[i % clones], pt_h, si_h, sl_h, out_h,
+                                      lse_h, staging, plan.workspace, plan.status)
+
+    e2e_steps = args.steps
+    for i in range(args.warmup):
+        e2e_step(i)
+    barrier()
+    e_begin, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e_begin.record()
+    for i in range(e2e_steps):
+        e2e_step(args.warmup + i)
+    e_end.record()
+    barrier()
+    e2e_ms_total = e_begin.elapsed_time(e_end)
+
+    # ---- reduce over ranks: slowest rank's time, all ranks' bytes ------------------------
+    times = torch.tensor([ms_total, e2e_ms_total], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    ms_total, e2e_ms_total = (float(x) for x in times.tolist())
+    ms_per_step = ms_total / args.steps
+    e2e_ms_per_step = e2e_ms_total / e2e_steps
+    value = world * kv_bytes / (ms_per_step * 1e-3) / 1e9
+    e2e_value = world * kv_bytes / (e2e_ms_per_step * 1e-3) / 1e9
+
+    if rank == 0:
+        peaks = _peaks()
+        kmean = statistics.mean(kern_ms)
+        achieved = kv_bytes / (kmean * 1e-3) / 1e9
+        khash = _kernel_source_hash()
+        tflops = flops / (kmean * 1e-3) / 1e12
+        line = {
+            "metric": "sparse MLA decode selected-KV bandwidth (us/step beside it)",
+            "value": round(value, 2), "unit": "GB/s", "us_per_step": round(ms_per_step * 1e3, 3),
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": round(ms_per_step, 6), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "config2 DeepSeek-R1-shaped decode: batch 32/GPU, 128 heads, d_qk 576, "
+                                   "d_v 512, ctx 32768, 64-token pages shuffled, 2112 selected tokens/request "
+                                   "(page 0 + last 512 + 24 middle pages), seed 1",
+                       "selected_tokens_per_gpu": w.selected_tokens, "kv_bytes_per_step_per_gpu": kv_bytes,
+                       "splits": plan.splits, "kernel": args.kernel,
+                       "l2": "cold: %d pool copies rotated (%.0f MB touched per cycle vs %.0f MB L2)"
+                             % (clones, clones * kv_bytes / 1e6, L2_BYTES / 1e6),
+                       "parallelism": "dp%d (independent requests, no collective)" % world},
+            "clocks": clocks,
+            "e2e": {"value": round(e2e_value, 2), "unit": "GB/s",
+                    "us_per_step": round(e2e_ms_per_step * 1e3, 3),
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "note": "omni_sparse_mla_decode_host: q, page_table, sel_idx, sel_len copied from pinned "
+                            "host memory and out, lse copied back every step; the KV cache is persistent "
+                            "device state"},
+            "gpu_launches": launches_per_step * args.steps,
+            "roofline": {"bound": "hbm", "achieved": round(achieved, 2), "peak": peaks["hbm"],
+                         "unit": "GB/s", "frac": round(achieved / peaks["hbm"], 4),
+                         "traffic": _recorded_traffic(khash), "peak_source": peaks["source"],
+                         "kernel": "sparse_mla_decode main kernel", "kernel_us_mean": round(kmean * 1e3, 3),
+                         "kernel_us_min": round(min(kern_ms) * 1e3, 3),
+                         "algorithmic_bytes_per_launch": kv_bytes,
+                         "tensor_tflops": round(tflops, 2),
+                         "tensor_frac_of_sustained": round(tflops / peaks["tc_sustained"], 4),
+                         "frac_of_nominal_8TBs": round(achieved / 8000.0, 4),
+                         "kernel_source_hash": khash},
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            s = _oracle_sample(w)
+            cpu_value = s["tokens"] * KV_ROW_BYTES / s["seconds"] / 1e9
+            line["cpu_baseline"] = {
+                "value": round(cpu_value, 5), "unit": "GB/s", "cores": s["cores"], "kind": "oracle",
+                "sample": "fp64 oracle on the first %d of %d requests (all 128 heads, %d selected tokens), "
+                          "%.1f s; full step extrapolates to %.0f us"
+                          % (s["requests"], w.batch, s["tokens"], s["seconds"],
+                             s["seconds"] / s["tokens"] * w.selected_tokens * 1e6)}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def reference_arm(args):
+    """The oracle as the reference implementation, timed on host cores on a bounded sample."""
+    import torch
+    from paper_2511_22481_b200 import workloads as W
+
+    # inputs of the same workload; a reduced pool is enough because only selected rows are read
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    w = W.config2_r1(dev)
+    per_step = max(2.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    times, tokens = [], 0
+    for i in range(args.warmup + args.steps):
+        s = _oracle_sample(w, target_s=per_step)
+        if i >= args.warmup:
+            times.append(s["seconds"])
+            tokens += s["tokens"]
+    total = sum(times)
+    value = tokens * KV_ROW_BYTES / total / 1e9
+    ms_per_step_full = total / tokens * w.selected_tokens * 1e3
+    line = {
+        "impl": "reference", "metric": "sparse MLA decode selected-KV bandwidth (us/step beside it)",
+        "value": round(value, 5), "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(ms_per_step_full, 3), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "config2 DeepSeek-R1-shaped decode (same as the CUDA arm); each step is a "
+                               "bounded sample of its requests, ms_per_step extrapolated to the full batch"},
+        "cpu_baseline": {"value": round(value, 5), "unit": "GB/s", "cores": s["cores"], "kind": "oracle",
+                         "sample": "%d requests x 128 heads per step, %.1f s per step" % (s["requests"], total / len(times))},
+        "e2e": {"value": round(value, 5), "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -1,0 +1,193 @@
+/*
+ * omni_mla.h -- C ABI of the sparse MLA decode library (B200 / sm_100a).
+ *
+ * The operation is the left-hand side of Eq. 1 of the paper's "OmniAttn: Problem
+ * Formulation": softmax(Q K_M^T * scale) V_M, attention restricted to a selected index
+ * set M, evaluated for one decode query per (request, head).  Eq. 2 (attention sink +
+ * recent tokens) is one producer of M; the library accepts any index list.  As the
+ * "Layer-wise Compression" paragraph requires, every head of a request shares one M,
+ * which is also what multi-latent attention needs: one latent row per token, K = all
+ * d_qk = 576 columns (512 latent + 64 rope), V = the first d_v = 512 columns.
+ *
+ * Conventions shared by every entry point
+ *   - Unless a parameter says "host", pointers are DEVICE pointers owned by the caller.
+ *     The library allocates no device memory and keeps no per-call state.
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*).  Errors the host
+ *     can see (null pointer, bad shape, misalignment, short workspace) are returned at once
+ *     and nothing is launched.
+ *   - Conditions only the device can see (a token position or page id out of range) never
+ *     trap: the offending entry is skipped (it contributes nothing), and if `device_status`
+ *     is non-NULL the word it points to is OR-ed with OMNI_DEV_BAD_INDEX.  A bounded wait
+ *     that runs out inside a kernel ORs OMNI_DEV_TIMEOUT and the affected outputs are
+ *     unspecified.  The caller zeroes the word and reads it back after synchronising.
+ *   - Inputs are never modified.  Distinct streams need distinct workspaces.
+ */
+#ifndef OMNI_MLA_H_
+#define OMNI_MLA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    OMNI_OK = 0,
+    OMNI_ERR_NULL = 1,      /* a required pointer is NULL                                  */
+    OMNI_ERR_SHAPE = 2,     /* unsupported or inconsistent sizes in the descriptor         */
+    OMNI_ERR_ALIGN = 3,     /* a pointer misses its required alignment                     */
+    OMNI_ERR_WORKSPACE = 4, /* workspace smaller than omni_sparse_mla_workspace_bytes()    */
+    OMNI_ERR_INDEX = 5,     /* reserved for host-side index checks                         */
+    OMNI_ERR_TIMEOUT = 6,   /* reserved                                                    */
+    OMNI_ERR_CUDA = 7,      /* a CUDA runtime / driver call failed (launch, tensor map)    */
+    OMNI_ERR_ARCH = 8       /* the current device is not compute capability 10.x           */
+} omni_status_t;
+
+/* bits OR-ed into *device_status by kernels */
+#define OMNI_DEV_BAD_INDEX 1
+#define OMNI_DEV_TIMEOUT 2
+
+/* descriptor flags */
+#define OMNI_FLAG_VALIDATE 1  /* run the index validation kernel before the decode kernel  */
+#define OMNI_FLAG_SIMT 2      /* use the plain-FMA bring-up kernel instead of tensor cores */
+
+/* Plain-data problem descriptor; copied at call time. */
+typedef struct {
+    int64_t num_pages;         /* pages in the pool, >= 1                                  */
+    int32_t batch;             /* B >= 1 requests                                          */
+    int32_t num_heads;         /* H in [1,128]                                             */
+    int32_t d_qk;              /* must be 576                                              */
+    int32_t d_v;               /* must be 512                                              */
+    int32_t page_size;         /* must be 64                                               */
+    int32_t max_pages_per_req; /* row stride of page_table, >= 1                           */
+    int32_t max_sel;           /* row stride of sel_idx, >= 1                              */
+    int32_t num_splits;        /* 0: library chooses; k >= 1: k split-KV partitions/request*/
+    float softmax_scale;       /* multiplies q.k before the softmax, e.g. 1/sqrt(192)      */
+    int32_t flags;             /* OMNI_FLAG_* bits                                         */
+} omni_mla_desc_t;
+
+/* Library version, major*1000 + minor. */
+int omni_version(void);
+
+/* Static, human-readable name of a status code. */
+const char *omni_status_string(omni_status_t status);
+
+/*
+ * Number of split-KV partitions per request the library will use for this descriptor on
+ * the current device (desc->num_splits if that is >= 1).  Returns 0 on a bad descriptor.
+ */
+int32_t omni_sparse_mla_num_splits(const omni_mla_desc_t *desc);
+
+/*
+ * Bytes of device workspace omni_sparse_mla_decode needs for this descriptor: room for the
+ * fp32 partial outputs and partial log-sum-exps of every (request, split).  Returns 0 on a
+ * bad descriptor.  The workspace must be 256-byte aligned; its contents need no
+ * initialisation and are overwritten.
+ */
+size_t omni_sparse_mla_workspace_bytes(const omni_mla_desc_t *desc);
+
+/*
+ * Decode-phase sparse MLA attention (Eq. 1 left-hand side over the index set of each
+ * request; split-KV partition and merge included).
+ *
+ * For request b, head h, with N = sel_len[b] and t_j = sel_idx[b][j] for j < N:
+ *     row_j = page_table[b][t_j / 64] * 64 + t_j % 64
+ *     x_j   = softmax_scale * sum_c q[b,h,c] * kv_cache[row_j][c]          c < 576
+ *     lse[b,h]   = ln sum_j exp(x_j)                                       (natural log)
+ *     out[b,h,d] = sum_j exp(x_j - lse[b,h]) * kv_cache[row_j][d]          d < 512
+ * N = 0 gives out = 0 and lse = -inf.  The order of sel_idx does not matter beyond
+ * rounding; repeated positions count once per occurrence.
+ *
+ *   q          bf16 [B, H, 576], contiguous, 16-byte aligned
+ *   kv_cache   bf16 [num_pages, 64, 576], contiguous, 128-byte aligned
+ *   page_table int32 [B, max_pages_per_req]: physical page id of each logical page
+ *   sel_idx    int32 [B, max_sel]: logical token positions; entries at j >= sel_len[b] are
+ *              never read as positions
+ *   sel_len    int32 [B], each in [0, max_sel]
+ *   out        bf16 [B, H, 512]            (written)
+ *   lse        fp32 [B, H]                 (written)
+ *   workspace  >= omni_sparse_mla_workspace_bytes(desc) bytes, 256-byte aligned
+ *   device_status  optional int32 word, see the conventions above; may be NULL
+ *
+ * Products are bf16 x bf16 accumulated in fp32; the softmax runs in fp32; the tensor-core
+ * path rounds the unnormalised weights to bf16 before the weighted sum.
+ */
+omni_status_t omni_sparse_mla_decode(const omni_mla_desc_t *desc, const void *q,
+                                     const void *kv_cache, const int32_t *page_table,
+                                     const int32_t *sel_idx, const int32_t *sel_len, void *out,
+                                     float *lse, void *workspace, size_t workspace_bytes,
+                                     int32_t *device_status, void *stream);
+
+/*
+ * Merge of split-KV partial results (the step that follows a partition of M into disjoint
+ * ranges; Eq. 1 is recovered exactly because softmax normalisers add):
+ *     lse[b,h]   = ln sum_s exp(part_lse[b,s,h])
+ *     out[b,h,d] = sum_s exp(part_lse[b,s,h] - lse[b,h]) * part_out[b,s,h,d]
+ *
+ *   max_splits  row stride S of the partial arrays, >= 1
+ *   part_out    fp32 [B, S, H, 512], each partial normalised by its own sum; 16-byte aligned
+ *   part_lse    fp32 [B, S, H]; -inf marks an empty partial (weight 0)
+ *   num_splits  int32 [B], each in [0, S], or NULL meaning S for every request
+ *   out         bf16 [B, H, 512]  (written);  lse fp32 [B, H] (written)
+ * If every partial of a (b,h) is empty the result is out = 0, lse = -inf.  Only batch,
+ * num_heads and d_v of the descriptor are used.
+ */
+omni_status_t omni_sparse_mla_combine(const omni_mla_desc_t *desc, int32_t max_splits,
+                                      const float *part_out, const float *part_lse,
+                                      const int32_t *num_splits, void *out, float *lse,
+                                      void *stream);
+
+/*
+ * Index contract check on the device: ORs OMNI_DEV_BAD_INDEX into *device_status if any
+ * sel_len[b] lies outside [0, max_sel], any read position is negative or beyond the page
+ * table row, or any page id it reaches lies outside [0, num_pages).  Launches one small
+ * kernel; reads nothing but the three index arrays.
+ */
+omni_status_t omni_sparse_mla_validate(const omni_mla_desc_t *desc, const int32_t *page_table,
+                                       const int32_t *sel_idx, const int32_t *sel_len,
+                                       int32_t *device_status, void *stream);
+
+/*
+ * Physical rows the decode kernel will read, for checking index handling bit for bit:
+ * rows[b][j] = row_j (int64) for j < sel_len[b], -1 elsewhere and for entries that violate
+ * the index contract.  rows is int64 [B, max_sel].
+ */
+omni_status_t omni_sparse_mla_resolve_rows(const omni_mla_desc_t *desc,
+                                           const int32_t *page_table, const int32_t *sel_idx,
+                                           const int32_t *sel_len, int64_t *rows, void *stream);
+
+/*
+ * Same operation as omni_sparse_mla_decode for callers whose per-step tensors live in HOST
+ * memory: q, page_table, sel_idx, sel_len are host pointers (pinned memory makes the copies
+ * asynchronous) and out / lse are host buffers that receive the result.  kv_cache stays a
+ * device pointer: the cache is state that persists across decode steps.
+ *
+ *   staging, staging_bytes   device scratch for the per-step tensors, at least
+ *                            omni_sparse_mla_host_staging_bytes(desc), 256-byte aligned
+ * The copies and kernels are all enqueued on `stream`; the host buffers may be read after the
+ * stream is synchronised.
+ */
+size_t omni_sparse_mla_host_staging_bytes(const omni_mla_desc_t *desc);
+omni_status_t omni_sparse_mla_decode_host(const omni_mla_desc_t *desc, const void *q_host,
+                                          const void *kv_cache,
+                                          const int32_t *page_table_host,
+                                          const int32_t *sel_idx_host,
+                                          const int32_t *sel_len_host, void *out_host,
+                                          float *lse_host, void *staging, size_t staging_bytes,
+                                          void *workspace, size_t workspace_bytes,
+                                          int32_t *device_status, void *stream);
+
+/*
+ * Profiling aid (no counterpart in the paper): when both events are non-NULL, every later
+ * omni_sparse_mla_decode call on this thread's process records `before` and `after`
+ * (cudaEvent_t passed as void*) on its stream immediately around the main decode kernel,
+ * excluding the validation and merge kernels, so a caller can time that kernel alone.
+ * Pass NULLs to switch it off.  Process-wide and not thread-safe: meant for benchmarks.
+ */
+void omni_sparse_mla_set_profile_events(void *before, void *after);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* OMNI_MLA_H_ */

@@ -1,0 +1,315 @@
+// Host side of the C ABI declared in omni_mla.h: argument checks, the split-KV plan,
+// workspace carving and kernel launches.  Nothing here allocates device memory.
+#include <cuda_runtime.h>
+
+#include <mutex>
+
+#include "combine.cuh"
+#include "common.cuh"
+#include "simt_decode.cuh"
+#include "tc_decode.cuh"
+
+namespace omni {
+namespace {
+
+constexpr int kMaxSplits = 32;
+
+cudaEvent_t g_profile_before = nullptr, g_profile_after = nullptr;
+
+struct DeviceInfo {
+    int sm_count = 0;
+    int cc_major = 0;
+    bool ok = false;
+};
+
+// Per-device facts, looked up once per device and process.
+const DeviceInfo &device_info()
+{
+    static DeviceInfo info[64];
+    static std::mutex mu;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+        static DeviceInfo none;
+        return none;
+    }
+    std::lock_guard<std::mutex> lock(mu);
+    if (!info[dev].ok) {
+        int sms = 0, major = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) == cudaSuccess) {
+            info[dev].sm_count = sms;
+            info[dev].cc_major = major;
+            info[dev].ok = true;
+        }
+    }
+    return info[dev];
+}
+
+bool desc_ok(const omni_mla_desc_t *d)
+{
+    return d && d->batch >= 1 && d->num_heads >= 1 && d->num_heads <= 128 && d->d_qk == kDqk &&
+           d->d_v == kDv && d->page_size == kPage && d->num_pages >= 1 &&
+           d->num_pages <= (int64_t)0x7fffffff / kPage && d->max_pages_per_req >= 1 &&
+           d->max_sel >= 1 && d->num_splits >= 0 && d->num_splits <= kMaxSplits;
+}
+
+bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+// Work units (CTAs) one split of one request occupies in the kernel that will run.
+int units_per_request(const omni_mla_desc_t *d)
+{
+    if (d->flags & OMNI_FLAG_SIMT)
+        return (d->num_heads + kSimtWarps * kSimtHeadsPerWarp - 1) / (kSimtWarps * kSimtHeadsPerWarp);
+    return (d->num_heads + kTcHeads - 1) / kTcHeads;
+}
+
+// Pick the number of split-KV partitions per request: the kernel's CTAs are laid out in
+// waves over the SMs, each CTA walking ceil(granules / S) 64-token granules, so minimise
+// waves * granules-per-CTA with a small charge per split for the merge.
+int choose_splits(const omni_mla_desc_t *d, int sm_count)
+{
+    if (d->num_splits >= 1) return d->num_splits;
+    if (sm_count <= 0) sm_count = 148;
+    const int granules = (d->max_sel + kTile - 1) / kTile;
+    const long units = (long)d->batch * units_per_request(d);
+    long best_cost = -1;
+    int best = 1;
+    for (int s = 1; s <= kMaxSplits && s <= granules; ++s) {
+        const long waves = (units * s + sm_count - 1) / sm_count;
+        const long per = (granules + s - 1) / s;
+        const long cost = waves * (per * 8 + 6) + (s > 1 ? 8 + s : 0);
+        if (best_cost < 0 || cost < best_cost) {
+            best_cost = cost;
+            best = s;
+        }
+    }
+    return best;
+}
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+size_t part_out_bytes(const omni_mla_desc_t *d, int splits)
+{
+    return align_up((size_t)d->batch * splits * d->num_heads * kDv * sizeof(float), 256);
+}
+
+size_t part_lse_bytes(const omni_mla_desc_t *d, int splits)
+{
+    return align_up((size_t)d->batch * splits * d->num_heads * sizeof(float), 256);
+}
+
+omni_status_t launch_combine(int batch, int heads, int max_splits, const float *part_out,
+                             const float *part_lse, const int32_t *num_splits, void *out,
+                             float *lse, cudaStream_t stream)
+{
+    combine_kernel<<<batch * heads, 128, 0, stream>>>(part_out, part_lse, num_splits, max_splits,
+                                                      heads, static_cast<__nv_bfloat16 *>(out), lse);
+    return cudaPeekAtLastError() == cudaSuccess ? OMNI_OK : OMNI_ERR_CUDA;
+}
+
+omni_status_t launch_resolve(const omni_mla_desc_t *d, const int32_t *page_table,
+                             const int32_t *sel_idx, const int32_t *sel_len, int64_t *rows,
+                             int32_t *status, cudaStream_t stream)
+{
+    dim3 grid((unsigned)min(64, (d->max_sel + 255) / 256), (unsigned)d->batch);
+    resolve_rows_kernel<<<grid, 256, 0, stream>>>(page_table, sel_idx, sel_len,
+                                                  d->max_pages_per_req, d->max_sel, d->num_pages,
+                                                  rows, status);
+    return cudaPeekAtLastError() == cudaSuccess ? OMNI_OK : OMNI_ERR_CUDA;
+}
+
+}  // namespace
+}  // namespace omni
+
+using namespace omni;
+
+extern "C" {
+
+int omni_version(void) { return 1000; }
+
+void omni_sparse_mla_set_profile_events(void *before, void *after)
+{
+    g_profile_before = static_cast<cudaEvent_t>(before);
+    g_profile_after = static_cast<cudaEvent_t>(after);
+}
+
+const char *omni_status_string(omni_status_t status)
+{
+    switch (status) {
+        case OMNI_OK: return "ok";
+        case OMNI_ERR_NULL: return "null pointer";
+        case OMNI_ERR_SHAPE: return "unsupported or inconsistent shape";
+        case OMNI_ERR_ALIGN: return "misaligned pointer";
+        case OMNI_ERR_WORKSPACE: return "workspace too small";
+        case OMNI_ERR_INDEX: return "index out of range";
+        case OMNI_ERR_TIMEOUT: return "device wait timed out";
+        case OMNI_ERR_CUDA: return "CUDA call failed";
+        case OMNI_ERR_ARCH: return "device is not compute capability 10.x";
+    }
+    return "unknown status";
+}
+
+int32_t omni_sparse_mla_num_splits(const omni_mla_desc_t *desc)
+{
+    if (!desc_ok(desc)) return 0;
+    return choose_splits(desc, device_info().sm_count);
+}
+
+size_t omni_sparse_mla_workspace_bytes(const omni_mla_desc_t *desc)
+{
+    if (!desc_ok(desc)) return 0;
+    const int s = choose_splits(desc, device_info().sm_count);
+    return part_out_bytes(desc, s) + part_lse_bytes(desc, s) + 256;
+}
+
+omni_status_t omni_sparse_mla_decode(const omni_mla_desc_t *desc, const void *q,
+                                     const void *kv_cache, const int32_t *page_table,
+                                     const int32_t *sel_idx, const int32_t *sel_len, void *out,
+                                     float *lse, void *workspace, size_t workspace_bytes,
+                                     int32_t *device_status, void *stream_)
+{
+    if (!desc || !q || !kv_cache || !page_table || !sel_idx || !sel_len || !out || !lse)
+        return OMNI_ERR_NULL;
+    if (!desc_ok(desc)) return OMNI_ERR_SHAPE;
+    if (!aligned(q, 16) || !aligned(kv_cache, 128) || !aligned(out, 16) || !aligned(lse, 4) ||
+        !aligned(page_table, 4) || !aligned(sel_idx, 4) || !aligned(sel_len, 4))
+        return OMNI_ERR_ALIGN;
+    const DeviceInfo &dev = device_info();
+    if (!dev.ok) return OMNI_ERR_CUDA;
+    if (dev.cc_major != 10) return OMNI_ERR_ARCH;
+    const int splits = choose_splits(desc, dev.sm_count);
+    const size_t need = part_out_bytes(desc, splits) + part_lse_bytes(desc, splits) + 256;
+    if (splits > 1) {
+        if (!workspace) return OMNI_ERR_NULL;
+        if (!aligned(workspace, 256)) return OMNI_ERR_ALIGN;
+        if (workspace_bytes < need) return OMNI_ERR_WORKSPACE;
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+
+    if (desc->flags & OMNI_FLAG_VALIDATE) {
+        omni_status_t st = launch_resolve(desc, page_table, sel_idx, sel_len, nullptr, device_status, stream);
+        if (st != OMNI_OK) return st;
+    }
+
+    DecodeParams p;
+    p.q = static_cast<const __nv_bfloat16 *>(q);
+    p.kv = static_cast<const __nv_bfloat16 *>(kv_cache);
+    p.page_table = page_table;
+    p.sel_idx = sel_idx;
+    p.sel_len = sel_len;
+    p.out = static_cast<__nv_bfloat16 *>(out);
+    p.lse = lse;
+    p.part_out = static_cast<float *>(workspace);
+    p.part_lse = splits > 1 ? reinterpret_cast<float *>(static_cast<char *>(workspace) + part_out_bytes(desc, splits))
+                            : nullptr;
+    p.status = device_status;
+    p.num_pages = desc->num_pages;
+    p.batch = desc->batch;
+    p.heads = desc->num_heads;
+    p.max_pages = desc->max_pages_per_req;
+    p.max_sel = desc->max_sel;
+    p.splits = splits;
+    p.scale_log2 = desc->softmax_scale * kLog2e;
+
+    if (g_profile_before && g_profile_after) cudaEventRecord(g_profile_before, stream);
+    if (desc->flags & OMNI_FLAG_SIMT) {
+        const int grid = desc->batch * splits * units_per_request(desc);
+        simt_decode_kernel<<<grid, kSimtWarps * 32, 0, stream>>>(p);
+        if (cudaPeekAtLastError() != cudaSuccess) return OMNI_ERR_CUDA;
+    } else {
+        omni_status_t st = launch_tc_decode(p, stream);
+        if (st != OMNI_OK) return st;
+    }
+    if (g_profile_before && g_profile_after) cudaEventRecord(g_profile_after, stream);
+    if (splits > 1)
+        return launch_combine(desc->batch, desc->num_heads, splits, p.part_out, p.part_lse, nullptr,
+                              out, lse, stream);
+    return OMNI_OK;
+}
+
+omni_status_t omni_sparse_mla_combine(const omni_mla_desc_t *desc, int32_t max_splits,
+                                      const float *part_out, const float *part_lse,
+                                      const int32_t *num_splits, void *out, float *lse,
+                                      void *stream)
+{
+    if (!desc || !part_out || !part_lse || !out || !lse) return OMNI_ERR_NULL;
+    if (desc->batch < 1 || desc->num_heads < 1 || desc->d_v != kDv || max_splits < 1)
+        return OMNI_ERR_SHAPE;
+    if (!aligned(part_out, 16) || !aligned(out, 8) || !aligned(part_lse, 4) || !aligned(lse, 4))
+        return OMNI_ERR_ALIGN;
+    return launch_combine(desc->batch, desc->num_heads, max_splits, part_out, part_lse, num_splits,
+                          out, lse, static_cast<cudaStream_t>(stream));
+}
+
+omni_status_t omni_sparse_mla_validate(const omni_mla_desc_t *desc, const int32_t *page_table,
+                                       const int32_t *sel_idx, const int32_t *sel_len,
+                                       int32_t *device_status, void *stream)
+{
+    if (!desc || !page_table || !sel_idx || !sel_len || !device_status) return OMNI_ERR_NULL;
+    if (!desc_ok(desc)) return OMNI_ERR_SHAPE;
+    return launch_resolve(desc, page_table, sel_idx, sel_len, nullptr, device_status,
+                          static_cast<cudaStream_t>(stream));
+}
+
+omni_status_t omni_sparse_mla_resolve_rows(const omni_mla_desc_t *desc,
+                                           const int32_t *page_table, const int32_t *sel_idx,
+                                           const int32_t *sel_len, int64_t *rows, void *stream)
+{
+    if (!desc || !page_table || !sel_idx || !sel_len || !rows) return OMNI_ERR_NULL;
+    if (!desc_ok(desc)) return OMNI_ERR_SHAPE;
+    return launch_resolve(desc, page_table, sel_idx, sel_len, rows, nullptr,
+                          static_cast<cudaStream_t>(stream));
+}
+
+size_t omni_sparse_mla_host_staging_bytes(const omni_mla_desc_t *desc)
+{
+    if (!desc_ok(desc)) return 0;
+    const size_t B = desc->batch, H = desc->num_heads;
+    return align_up(B * H * kDqk * 2, 256) + align_up(B * desc->max_pages_per_req * 4, 256) +
+           align_up(B * desc->max_sel * 4, 256) + align_up(B * 4, 256) +
+           align_up(B * H * kDv * 2, 256) + align_up(B * H * 4, 256);
+}
+
+omni_status_t omni_sparse_mla_decode_host(const omni_mla_desc_t *desc, const void *q_host,
+                                          const void *kv_cache,
+                                          const int32_t *page_table_host,
+                                          const int32_t *sel_idx_host,
+                                          const int32_t *sel_len_host, void *out_host,
+                                          float *lse_host, void *staging, size_t staging_bytes,
+                                          void *workspace, size_t workspace_bytes,
+                                          int32_t *device_status, void *stream_)
+{
+    if (!desc || !q_host || !kv_cache || !page_table_host || !sel_idx_host || !sel_len_host ||
+        !out_host || !lse_host || !staging)
+        return OMNI_ERR_NULL;
+    if (!desc_ok(desc)) return OMNI_ERR_SHAPE;
+    if (!aligned(staging, 256)) return OMNI_ERR_ALIGN;
+    if (staging_bytes < omni_sparse_mla_host_staging_bytes(desc)) return OMNI_ERR_WORKSPACE;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const size_t B = desc->batch, H = desc->num_heads;
+    const size_t nq = B * H * kDqk * 2, npt = B * desc->max_pages_per_req * 4,
+                 nsi = B * desc->max_sel * 4, nsl = B * 4, nout = B * H * kDv * 2, nlse = B * H * 4;
+    char *base = static_cast<char *>(staging);
+    char *dq = base;
+    char *dpt = dq + align_up(nq, 256);
+    char *dsi = dpt + align_up(npt, 256);
+    char *dsl = dsi + align_up(nsi, 256);
+    char *dout = dsl + align_up(nsl, 256);
+    char *dlse = dout + align_up(nout, 256);
+    if (cudaMemcpyAsync(dq, q_host, nq, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+        cudaMemcpyAsync(dpt, page_table_host, npt, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+        cudaMemcpyAsync(dsi, sel_idx_host, nsi, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+        cudaMemcpyAsync(dsl, sel_len_host, nsl, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        return OMNI_ERR_CUDA;
+    omni_status_t st = omni_sparse_mla_decode(
+        desc, dq, kv_cache, reinterpret_cast<int32_t *>(dpt), reinterpret_cast<int32_t *>(dsi),
+        reinterpret_cast<int32_t *>(dsl), dout, reinterpret_cast<float *>(dlse), workspace,
+        workspace_bytes, device_status, stream_);
+    if (st != OMNI_OK) return st;
+    if (cudaMemcpyAsync(out_host, dout, nout, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+        cudaMemcpyAsync(lse_host, dlse, nlse, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+        return OMNI_ERR_CUDA;
+    return OMNI_OK;
+}
+
+}  // extern "C"

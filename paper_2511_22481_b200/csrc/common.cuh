@@ -1,0 +1,63 @@
+// Shared device-side definitions of the sparse MLA decode kernels (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "omni_mla.h"
+
+namespace omni {
+
+constexpr int kDqk = 576;        // latent row: 512 "nope" + 64 rope columns, all used as K
+constexpr int kDv = 512;         // the first 512 columns of the same row are V
+constexpr int kPage = 64;        // tokens per page
+constexpr int kTile = 64;        // tokens per split-KV granule (split boundaries fall on these)
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+// Everything a kernel needs to find its data; passed by value.
+struct DecodeParams {
+    const __nv_bfloat16 *q;        // [B, H, 576]
+    const __nv_bfloat16 *kv;       // [num_pages * 64, 576]
+    const int32_t *page_table;     // [B, max_pages]
+    const int32_t *sel_idx;        // [B, max_sel]
+    const int32_t *sel_len;        // [B]
+    __nv_bfloat16 *out;            // [B, H, 512]
+    float *lse;                    // [B, H]
+    float *part_out;               // [B, S, H, 512]  (S > 1 only)
+    float *part_lse;               // [B, S, H]
+    int32_t *status;               // may be null
+    int64_t num_pages;
+    int32_t batch, heads, max_pages, max_sel, splits;
+    float scale_log2;              // softmax_scale * log2(e)
+};
+
+// Token range [begin, end) of split s of a request with n selected tokens: the n tokens are
+// cut into 64-token granules and the granules are dealt out in contiguous, equal runs.
+__device__ __forceinline__ void split_range(int n, int splits, int s, int &begin, int &end)
+{
+    const int granules = (n + kTile - 1) / kTile;
+    const int per = (granules + splits - 1) / splits;
+    begin = min(n, s * per * kTile);
+    end = min(n, (s + 1) * per * kTile);
+}
+
+// Logical token position -> physical pool row, or -1 if the entry breaks the index contract.
+__device__ __forceinline__ int64_t resolve_row(const int32_t *page_table_row, int32_t t,
+                                               int32_t max_pages, int64_t num_pages)
+{
+    if (t < 0) return -1;
+    const int32_t lp = t / kPage;
+    if (lp >= max_pages) return -1;
+    const int32_t page = __ldg(page_table_row + lp);
+    if (page < 0 || (int64_t)page >= num_pages) return -1;
+    return (int64_t)page * kPage + (t % kPage);
+}
+
+__device__ __forceinline__ void flag_status(int32_t *status, int32_t bits)
+{
+    if (status != nullptr) atomicOr(status, bits);
+}
+
+}  // namespace omni

@@ -1,0 +1,104 @@
+"""The C-ABI library loads, exports every function the header declares, and rejects bad
+arguments on the host before touching a device (no compute calls: runs without a GPU)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2511_22481_b200 import binding as B
+from paper_2511_22481_b200 import build as builder
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    builder.build()
+    return B.load()
+
+
+def _declared_functions():
+    names = set()
+    inc = os.path.join(ROOT, "include")
+    for fn in os.listdir(inc):
+        text = open(os.path.join(inc, fn)).read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        names.update(re.findall(r"\b(omni_[a-z0-9_]+)\s*\(", text))
+    return names
+
+
+def test_every_declared_function_is_exported(lib):
+    declared = _declared_functions()
+    assert declared == set(B.EXPORTS)
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+def test_version_and_status_strings(lib):
+    assert B.omni_version() >= 1000
+    seen = {B.status_string(c) for c in range(9)}
+    assert len(seen) == 9 and "ok" in seen
+
+
+def test_descriptor_mirror_has_the_c_layout():
+    assert ctypes.sizeof(B.OmniDesc) == 48
+    assert B.OmniDesc.num_pages.offset == 0 and B.OmniDesc.batch.offset == 8
+    assert B.OmniDesc.softmax_scale.offset == 40 and B.OmniDesc.flags.offset == 44
+
+
+def _desc(**kw):
+    args = dict(batch=2, num_heads=128, num_pages=8, max_pages_per_req=4, max_sel=256, softmax_scale=0.1)
+    args.update(kw)
+    return B.make_desc(**args)
+
+
+def test_bad_descriptors_are_rejected(lib):
+    for kw in (dict(batch=0), dict(num_heads=0), dict(num_heads=129), dict(d_qk=512), dict(d_v=576),
+               dict(page_size=128), dict(num_pages=0), dict(max_sel=0), dict(num_splits=-1),
+               dict(num_splits=1000), dict(max_pages_per_req=0)):
+        d = _desc(**kw)
+        assert B.omni_sparse_mla_workspace_bytes(d) == 0, kw
+        assert B.omni_sparse_mla_num_splits(d) == 0, kw
+        code = lib.omni_sparse_mla_decode(ctypes.byref(d), *([ctypes.c_void_p(256)] * 7),
+                                          ctypes.c_void_p(256), 1 << 30, None, None)
+        assert code == 2, kw                                 # OMNI_ERR_SHAPE
+
+
+def test_null_and_misaligned_pointers_are_rejected(lib):
+    d = _desc()
+    ok = ctypes.c_void_p(4096)
+    for missing in range(7):
+        ptrs = [ok] * 7
+        ptrs[missing] = None
+        assert lib.omni_sparse_mla_decode(ctypes.byref(d), *ptrs, ok, 1 << 30, None, None) == 1
+    assert lib.omni_sparse_mla_decode(None, *([ok] * 7), ok, 1 << 30, None, None) == 1
+    ptrs = [ok] * 7
+    ptrs[1] = ctypes.c_void_p(4096 + 64)                      # kv_cache must be 128-byte aligned
+    assert lib.omni_sparse_mla_decode(ctypes.byref(d), *ptrs, ok, 1 << 30, None, None) == 3
+    ptrs = [ok] * 7
+    ptrs[0] = ctypes.c_void_p(4096 + 2)                       # q must be 16-byte aligned
+    assert lib.omni_sparse_mla_decode(ctypes.byref(d), *ptrs, ok, 1 << 30, None, None) == 3
+    assert lib.omni_sparse_mla_combine(ctypes.byref(d), 0, ok, ok, None, ok, ok, None) == 2
+    assert lib.omni_sparse_mla_combine(ctypes.byref(d), 2, None, ok, None, ok, ok, None) == 1
+    assert lib.omni_sparse_mla_validate(ctypes.byref(d), ok, ok, ok, None, None) == 1
+    assert lib.omni_sparse_mla_resolve_rows(ctypes.byref(d), ok, ok, ok, None, None) == 1
+    assert lib.omni_sparse_mla_decode_host(ctypes.byref(d), *([ok] * 7), None, 0, ok, 0, None, None) == 1
+
+
+def test_workspace_grows_with_forced_splits(lib):
+    a = B.omni_sparse_mla_workspace_bytes(_desc(num_splits=1))
+    b = B.omni_sparse_mla_workspace_bytes(_desc(num_splits=4))
+    assert 0 < a < b and b >= 2 * 4 * 128 * 513 * 4
+    assert B.omni_sparse_mla_num_splits(_desc(num_splits=4)) == 4
+    assert B.omni_sparse_mla_host_staging_bytes(_desc()) >= 2 * 128 * (576 + 512) * 2
+
+
+def test_binding_refuses_cpu_tensors_for_device_arguments():
+    import torch
+    d = _desc()
+    t = torch.zeros(4, dtype=torch.bfloat16)
+    with pytest.raises(ValueError):
+        B._ptr(t, torch.bfloat16, "cuda", "q")
+    with pytest.raises(TypeError):
+        B._ptr(t, torch.int32, "cpu", "sel_idx")

@@ -1,0 +1,230 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle, element by element on
+small problems and on sampled (request, head) rows at the full benchmark sizes."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2511_22481_b200 import binding as B
+from paper_2511_22481_b200 import workloads as W
+from parity import check_workload, compare, oracle_subset, run_gpu
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+IMPLS = {"simt": B.OMNI_FLAG_SIMT, "tc": 0}
+
+
+@pytest.fixture(params=list(IMPLS))
+def flags(request):
+    return IMPLS[request.param]
+
+
+def _custom(name, seed, heads, ctx_pages, sel_lists, shuffle=True):
+    """Workload from explicit per-request selection lists."""
+    rng = np.random.default_rng(seed)
+    tables = W._shuffled_tables(rng, ctx_pages, shuffle)
+    return W._pack(name, seed, heads, list(ctx_pages), tables,
+                   [np.asarray(s, dtype=np.int32) for s in sel_lists], DEV, dict(kind="custom"))
+
+
+# ------------------------------------------------------------------ small, every element
+
+def test_config1_tiny(flags):
+    stats, plan = check_workload(W.config1_tiny(DEV), flags, what="config1")
+    assert stats["max_abs"] < 1e-3
+
+
+@pytest.mark.parametrize("splits", [1, 2, 3, 7])
+def test_forced_splits_including_empty_ones(flags, splits):
+    w = W.page_sparse("small", 40, 3, 128, [8, 5, 16], 2, [1, 0, 3], DEV)
+    check_workload(w, flags, num_splits=splits, what="splits=%d" % splits)
+
+
+def test_ragged_lengths_and_tails(flags):
+    rng = np.random.default_rng(41)
+    lens = [0, 1, 2, 63, 64, 65, 127, 129, 300, 513]
+    sels = [rng.permutation(16 * 64)[:n] for n in lens]
+    w = _custom("ragged_tails", 41, 128, [16] * len(lens), sels)
+    for s in (0, 1, 4):
+        stats, plan = check_workload(w, flags, num_splits=s, what="ragged tails S=%d" % s)
+        assert torch.all(plan.out[0] == 0) and torch.all(torch.isneginf(plan.lse[0]))
+
+
+@pytest.mark.parametrize("heads", [1, 16, 48, 64, 80, 128])
+def test_head_counts(flags, heads):
+    w = W.token_topk("heads%d" % heads, 42, 2, heads, 8, 200, DEV)
+    check_workload(w, flags, what="H=%d" % heads)
+
+
+def test_token_level_unsorted_selection(flags):
+    w = W.config4_topk(DEV, batch=3, ctx_pages=64, k=777)
+    check_workload(w, flags, num_splits=3, what="topk small")
+
+
+def test_dense_selection_equals_oracle(flags):
+    w = W.dense("dense_small", 43, 2, 128, 12, DEV)
+    check_workload(w, flags, what="dense small")
+
+
+def test_same_bits_on_repeat(flags):
+    w = W.config4_topk(DEV, batch=2, ctx_pages=32, k=500)
+    a = run_gpu(w, flags)
+    o1, l1 = a.out.clone(), a.lse.clone()
+    b = run_gpu(w, flags, plan=a)
+    assert torch.equal(o1, b.out) and torch.equal(l1, b.lse)
+
+
+# ------------------------------------------------------------------ index handling, bit exact
+
+def test_resolved_rows_match_oracle_bit_for_bit():
+    for w in (W.config1_tiny(DEV), W.config4_topk(DEV, batch=4, ctx_pages=128, k=1000),
+              W.config3_ragged(DEV, batch=6)):
+        desc = B.make_desc(w.batch, w.heads, w.num_pages, w.max_pages_per_req, w.max_sel, w.scale)
+        rows = torch.empty((w.batch, w.max_sel), dtype=torch.int64, device=DEV)
+        B.omni_sparse_mla_resolve_rows(desc, w.page_table, w.sel_idx, w.sel_len, rows)
+        torch.cuda.synchronize()
+        ref = oracle.resolve_rows(w.page_table.cpu().numpy(), w.sel_idx.cpu().numpy(),
+                                  w.sel_len.cpu().numpy(), w.page_size, w.num_pages)
+        assert np.array_equal(rows.cpu().numpy(), ref)
+
+
+@pytest.mark.parametrize("hi", [0, 1])
+def test_histogram_of_rows_read_is_exact(flags, hi):
+    # q = 0 -> uniform weights 1/N (N a power of two); one-hot value rows make N*out an exact
+    # histogram of the physical rows that were read.
+    n_pages, N = 24, 512
+    w = W.token_topk("hist", 44, 2, 128, n_pages, N, DEV)
+    w.q.zero_()
+    rows_all = torch.arange(n_pages * 2 * 64, device=DEV)
+    col = (rows_all % 512) if hi == 0 else ((rows_all // 512) % 512)
+    w.kv_cache.zero_()
+    w.kv_cache.view(-1, 576)[rows_all, col] = 1.0
+    for splits in (1, 4):
+        plan = run_gpu(w, flags, num_splits=splits)
+        ref_out, ref_lse, _ = oracle_subset(w)
+        got = plan.out.to(torch.float64).cpu().numpy() * N
+        assert np.array_equal(got, ref_out * N)
+        assert np.abs(plan.lse.cpu().numpy() - math.log(N)).max() < 1e-5
+
+
+def test_spiked_row_comes_back_bit_exact(flags):
+    w = W.token_topk("spike", 45, 2, 128, 16, 300, DEV)
+    w.kv_cache[..., 512:] = 0
+    w.q[..., 512:] = 0
+    j = 123
+    rows = oracle.resolve_rows(w.page_table.cpu().numpy(), w.sel_idx.cpu().numpy(),
+                               w.sel_len.cpu().numpy(), 64, w.num_pages)
+    w.q[..., 575] = 64.0
+    for b in range(2):
+        w.kv_cache.view(-1, 576)[int(rows[b, j]), 575] = 64.0
+    plan = run_gpu(w, flags, num_splits=2)
+    for b in range(2):
+        want = w.kv_cache.view(-1, 576)[int(rows[b, j]), :512]
+        assert torch.equal(plan.out[b], want.expand(128, 512))
+
+
+def test_single_token_returns_its_row_exactly(flags):
+    w = _custom("one", 46, 128, [4], [[77]])
+    plan = run_gpu(w, flags)
+    row = int(w.page_table[0, 1].item()) * 64 + 13
+    assert torch.equal(plan.out[0], w.kv_cache.view(-1, 576)[row, :512].expand(128, 512))
+    ref_out, ref_lse, _ = oracle_subset(w)
+    assert np.abs(plan.lse.cpu().numpy() - ref_lse).max() < 1e-4
+
+
+def test_out_of_range_entries_are_flagged_and_skipped(flags):
+    rng = np.random.default_rng(47)
+    sel = rng.permutation(8 * 64)[:200].astype(np.int32)
+    w = _custom("bad", 47, 128, [8], [sel])
+    good = _custom("good", 47, 128, [8], [np.delete(sel, [5, 150])])
+    bad_idx = w.sel_idx.clone()
+    bad_idx[0, 5] = -3
+    bad_idx[0, 150] = 8 * 64 + 1
+    w.sel_idx = bad_idx
+    plan = run_gpu(w, flags)
+    assert int(plan.status.item()) & B.OMNI_DEV_BAD_INDEX
+    ref_out, ref_lse, _ = oracle_subset(good)
+    compare(plan.out.cpu(), plan.lse.cpu(), ref_out, ref_lse, "skip bad entries")
+    desc = B.make_desc(1, 128, w.num_pages, w.max_pages_per_req, w.max_sel, w.scale)
+    st = torch.zeros(1, dtype=torch.int32, device=DEV)
+    B.omni_sparse_mla_validate(desc, w.page_table, w.sel_idx, w.sel_len, st)
+    assert int(st.item()) == B.OMNI_DEV_BAD_INDEX
+    st.zero_()
+    B.omni_sparse_mla_validate(desc, good.page_table, good.sel_idx, good.sel_len, st)
+    assert int(st.item()) == 0
+
+
+# ------------------------------------------------------------------ combine entry point
+
+def test_combine_entry_point_matches_oracle():
+    g = torch.Generator(device="cpu").manual_seed(48)
+    Bn, S, H = 3, 5, 16
+    po = torch.randn((Bn, S, H, 512), generator=g)
+    pl = torch.randn((Bn, S, H), generator=g) * 3
+    pl[0, 2] = -math.inf
+    pl[1, :, 3] = -math.inf
+    ns = torch.tensor([5, 4, 0], dtype=torch.int32)
+    ref_out, ref_lse = oracle.splitkv_combine(po.numpy().astype(np.float64), pl.numpy().astype(np.float64), ns.numpy())
+    desc = B.make_desc(Bn, H, 1, 1, 1, 1.0)
+    out = torch.empty((Bn, H, 512), dtype=torch.bfloat16, device=DEV)
+    lse = torch.empty((Bn, H), dtype=torch.float32, device=DEV)
+    B.omni_sparse_mla_combine(desc, S, po.to(DEV), pl.to(DEV), ns.to(DEV), out, lse)
+    torch.cuda.synchronize()
+    got = out.to(torch.float64).cpu().numpy()
+    assert np.abs(got - ref_out).max() <= 2 ** -8 * np.abs(ref_out).max()       # bf16 output rounding
+    gl = lse.cpu().numpy().astype(np.float64)
+    assert np.array_equal(np.isneginf(gl), np.isneginf(ref_lse))
+    fin = np.isfinite(ref_lse)
+    assert np.abs(gl[fin] - ref_lse[fin]).max() < 1e-5
+    assert torch.all(out[2] == 0) and torch.all(out[1, 3] == 0)
+
+
+# ------------------------------------------------------------------ host-buffer entry point
+
+def test_host_buffer_entry_point(flags):
+    w = W.config4_topk(DEV, batch=2, ctx_pages=32, k=300)
+    desc = B.make_desc(w.batch, w.heads, w.num_pages, w.max_pages_per_req, w.max_sel, w.scale, flags=flags)
+    staging = torch.empty(B.omni_sparse_mla_host_staging_bytes(desc), dtype=torch.uint8, device=DEV)
+    ws = torch.empty(B.omni_sparse_mla_workspace_bytes(desc), dtype=torch.uint8, device=DEV)
+    pin = lambda t: t.cpu().pin_memory()
+    out_h = torch.empty((w.batch, w.heads, 512), dtype=torch.bfloat16).pin_memory()
+    lse_h = torch.empty((w.batch, w.heads), dtype=torch.float32).pin_memory()
+    B.omni_sparse_mla_decode_host(desc, pin(w.q), w.kv_cache, pin(w.page_table), pin(w.sel_idx),
+                                  pin(w.sel_len), out_h, lse_h, staging, ws)
+    torch.cuda.synchronize()
+    ref_out, ref_lse, _ = oracle_subset(w)
+    compare(out_h, lse_h, ref_out, ref_lse, "host entry point")
+
+
+# ------------------------------------------------------------------ full benchmark sizes, sampled
+
+def test_config2_full_size_sampled(flags):
+    w = W.config2_r1(DEV)
+    check_workload(w, flags, reqs=[0, 13, 31], heads=[0, 63, 64, 127], what="config2")
+
+
+def test_config2_2048_variant(flags):
+    w = W.config2_r1(DEV, middle_pages=23)
+    check_workload(w, flags, reqs=[7], heads=[1, 100], what="config2/2048")
+
+
+def test_config3_ragged_full_size_sampled(flags):
+    w = W.config3_ragged(DEV)
+    sl = w.sel_len.cpu().numpy()
+    reqs = sorted({int(sl.argmin()), int(sl.argmax()), 0, 127})
+    check_workload(w, flags, reqs=reqs, heads=[0, 77, 127], what="config3")
+
+
+def test_config4_topk_full_size_sampled(flags):
+    w = W.config4_topk(DEV)
+    check_workload(w, flags, reqs=[0, 15], heads=[0, 64, 127], what="config4")
+
+
+def test_config5_cells_sampled():
+    for batch, n in ((1, 512), (8, 8192), (32, 2048)):
+        w = W.config5_cell(batch, n, DEV)
+        check_workload(w, 0, reqs=[batch - 1], heads=[5, 126], what="config5 B%d N%d" % (batch, n))
+    w = W.config5_cell(1, 512, DEV, dense_variant=True)
+    check_workload(w, 0, reqs=[0], heads=[9], what="config5 dense B1")
