@@ -122,7 +122,7 @@ def _oracle_sample(w, target_s=15.0, max_requests=None):
         sl = w.sel_len[reqs].cpu().numpy()
         rows = oracle.resolve_rows(pt, si, sl, w.page_size, w.num_pages)
         gather = torch.from_numpy(np.where(rows < 0, 0, rows)).to(w.kv_cache.device)
-        krows = w.kv_cache.view(-1, w.d_qk)[gather.view(-1)].view(len(reqs), -1, w.d_qk).cpu()
+        krows = w.kv_cache.view(-1, w.d_qk)[gather.view(-1)].view(rows.shape[0], -1, w.d_qk).cpu()
         q = w.q[reqs].cpu()
         t0 = time.perf_counter()
         oracle.attend_rows(q, krows, sl, w.d_v, w.scale)

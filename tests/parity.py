@@ -2,10 +2,14 @@
 same (request, head) results with the CPU oracle on the same bits, and compare.
 
 Tolerances (bf16 inputs, fp32 accumulation, bf16 output):
-  * out: max |gpu - oracle| <= 2e-3 over all elements, and per (request, head) row
-         max_d |gpu - oracle| <= 1e-2 * max_d |oracle|   (element-wise relative error is
-         meaningless next to zero crossings, so the relative bound is taken against the row's
-         largest magnitude)
+  * out: every element |gpu - oracle| <= 2e-3 + 2^-8 * |oracle|.  The second term is one bf16
+         ulp of the value: the output format alone rounds by up to half of it, which exceeds
+         2e-3 once |out| >= 0.5 (selections of one or two tokens).  At the benchmark shapes
+         |out| < 0.1 and the tests also assert the plain max |gpu - oracle| <= 2e-3
+         (``strict_abs``).
+  * out: per (request, head) row max_d |gpu - oracle| <= 1e-2 * max_d |oracle| (element-wise
+         relative error is meaningless next to zero crossings, so the relative bound is taken
+         against the row's largest magnitude)
   * lse: |gpu - oracle| <= 2e-3
 """
 from __future__ import annotations
@@ -48,7 +52,7 @@ def oracle_subset(w, reqs=None, heads=None):
     return out, lse, rows
 
 
-def compare(gpu_out, gpu_lse, ref_out, ref_lse, what=""):
+def compare(gpu_out, gpu_lse, ref_out, ref_lse, what="", strict_abs=False):
     g = gpu_out.to(torch.float64).cpu().numpy()
     gl = gpu_lse.to(torch.float64).cpu().numpy()
     err = np.abs(g - ref_out)
@@ -56,17 +60,21 @@ def compare(gpu_out, gpu_lse, ref_out, ref_lse, what=""):
     row_err = err.max(axis=-1)
     rel = np.where(row_ref > 0, row_err / np.where(row_ref > 0, row_ref, 1.0), row_err)
     both_inf = np.isneginf(gl) & np.isneginf(ref_lse)
-    lse_err = np.where(both_inf, 0.0, np.abs(gl - ref_lse))
+    with np.errstate(invalid="ignore"):
+        lse_err = np.where(both_inf, 0.0, np.abs(gl - ref_lse))
     stats = dict(max_abs=float(err.max(initial=0.0)), max_row_rel=float(rel.max(initial=0.0)),
                  max_lse=float(np.nan_to_num(lse_err, nan=np.inf).max(initial=0.0)))
     assert np.all(np.isfinite(g)), what + ": non-finite output"
-    assert stats["max_abs"] <= ABS_TOL, "%s: max abs err %.3e" % (what, stats["max_abs"])
+    excess = float((err - (ABS_TOL + 2.0 ** -8 * np.abs(ref_out))).max(initial=-1.0))
+    assert excess <= 0.0, "%s: abs err exceeds 2e-3 + ulp by %.3e (max abs %.3e)" % (what, excess, stats["max_abs"])
+    if strict_abs:
+        assert stats["max_abs"] <= ABS_TOL, "%s: max abs err %.3e" % (what, stats["max_abs"])
     assert stats["max_row_rel"] <= REL_TOL, "%s: max row-relative err %.3e" % (what, stats["max_row_rel"])
     assert stats["max_lse"] <= LSE_TOL, "%s: max lse err %.3e" % (what, stats["max_lse"])
     return stats
 
 
-def check_workload(w, flags=0, num_splits=0, reqs=None, heads=None, what=""):
+def check_workload(w, flags=0, num_splits=0, reqs=None, heads=None, what="", strict_abs=False):
     plan = run_gpu(w, flags=flags, num_splits=num_splits)
     assert int(plan.status.item()) == 0, what + ": device status %d" % int(plan.status.item())
     ref_out, ref_lse, _ = oracle_subset(w, reqs, heads)
@@ -74,4 +82,4 @@ def check_workload(w, flags=0, num_splits=0, reqs=None, heads=None, what=""):
     h = torch.arange(w.heads) if heads is None else torch.tensor(list(heads))
     g = plan.out.cpu()[r][:, h]
     gl = plan.lse.cpu()[r][:, h]
-    return compare(g, gl, ref_out, ref_lse, what), plan
+    return compare(g, gl, ref_out, ref_lse, what, strict_abs), plan
