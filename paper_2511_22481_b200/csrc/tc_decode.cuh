@@ -1,7 +1,606 @@
-// placeholder until the tensor-core kernel lands
+// Tensor-core decode kernel for sm_100a: TMA row gather through the page table, tcgen05 MMAs
+// with fp32 accumulators in tensor memory, fp32 online softmax.
+//
+// One CTA owns 64 heads of one (request, split) and walks the split's selected tokens in
+// 64-token tiles:
+//   warp 0      producer: resolves token positions to pool rows and gathers the rows with
+//               TMA (4 rows per instruction) into a 2-stage ring of 128B-swizzled tiles
+//   warp 1      MMA issuer: S = Q K^T (M=64 heads, N=64 tokens, K=576) and O += P V
+//               (M=64, N=512, K=64); owns the tensor-memory allocation
+//   warps 2-5   softmax: read S from tensor memory, keep the running reference maximum and
+//               row sums, write P (bf16) to shared memory, rescale O when the reference
+//               moves, and run the epilogue
+//
+// Tensor-memory map (an M=64 accumulator occupies lanes 0-15 of each 32-lane quarter, so two
+// accumulators share a column range at lane offsets 0 and 16):
+//   columns   0..255  O   (lane offset 0: value columns 0..255, lane offset 16: 256..511)
+//   columns 256..287  S buffer 0 (lane offset 0: tokens 0..31 of the tile, 16: tokens 32..63)
+//   columns 288..319  S buffer 1
+// so every softmax thread owns half a row: lane l of a warp serves head row 16*(warp%4)+l%16
+// and the token / value-column half l/16.
 #pragma once
+
+#include <cuda.h>
+
 #include "common.cuh"
+
 namespace omni {
-constexpr int kTcHeads = 64;
-inline omni_status_t launch_tc_decode(const DecodeParams &, cudaStream_t) { return OMNI_ERR_CUDA; }
+
+constexpr int kTcHeads = 64;                       // heads per CTA (MMA M)
+constexpr int kTcThreads = 192;
+constexpr int kPanelBytes = kTile * 128;           // 64 rows x 64 bf16 columns, 128B-swizzled
+constexpr int kPanels = kDqk / 64;                 // 9 column panels per latent row
+constexpr int kTileBytes = kPanels * kPanelBytes;  // 73,728
+constexpr int kStages = 2;
+constexpr int kPBytes = kTcHeads * kTile * 2;      // 8,192
+constexpr int kSmemQ = 0;
+constexpr int kSmemKV = kSmemQ + kTileBytes;
+constexpr int kSmemP = kSmemKV + kStages * kTileBytes;
+constexpr int kSmemCtl = kSmemP + kPBytes;
+constexpr int kSmemCtlBytes = 256;
+constexpr int kTcSmemBytes = kSmemCtl + kSmemCtlBytes + 1024;  // + slack for 1024B alignment
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kColO = 0, kColS = 256;
+constexpr uint32_t kLane16 = 16u << 16;
+constexpr float kRescaleThreshold = 8.f;           // log2 units the reference max may lag
+constexpr long long kWaitCycles = 1ll << 31;         // about a second of SM clocks per wait
+
+struct TcControl {
+    uint64_t q_full;
+    uint64_t kv_full[kStages];
+    uint64_t kv_empty[kStages];
+    uint64_t s_full[2];
+    uint64_t s_empty[2];
+    uint64_t p_full;
+    uint64_t pv_done;
+    uint64_t valid_mask[kStages];
+    uint32_t tmem_base;
+    uint32_t abort;
+};
+static_assert(sizeof(TcControl) <= kSmemCtlBytes, "control block too large");
+
+// ---------------------------------------------------------------------------------------
+// thin PTX wrappers
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p)
+{
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+                 : "memory");
+}
+
+// Bounded wait on a phase parity; false if about a second passed without the phase completing.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity)
+{
+    const uint32_t addr = smem_u32(bar);
+    const long long start = clock64();
+    for (uint32_t it = 0;; ++it) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(addr), "r"(parity)
+            : "memory");
+        if (done) return true;
+        if ((it & 63u) == 63u && clock64() - start > kWaitCycles) return false;
+    }
+}
+
+__device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap *map, uint64_t *bar, int col,
+                                            int r0, int r1, int r2, int r3)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cta.global.tile::gather4.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+        ::"r"(dst), "l"(map), "r"(col), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(smem_u32(bar))
+        : "memory");
+}
+
+__device__ __forceinline__ void tma_box2d(uint32_t dst, const CUtensorMap *map, uint64_t *bar, int col, int row)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cta.global.tile.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(col), "r"(row), "r"(smem_u32(bar))
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint64_t *bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+
+// D[tmem] (+)= A[smem] * B[smem], bf16 inputs, fp32 accumulate.
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                       uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_st32(uint32_t taddr, const uint32_t (&v)[32])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]),
+          "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]),
+          "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// Shared-memory operand descriptor, 128-byte swizzle.  Field layout (bits): [0,14) start
+// address >> 4, [16,30) leading byte offset >> 4, [32,46) stride byte offset >> 4,
+// [46,48) descriptor version (1 on sm_100), [61,64) swizzle mode (2 = 128 B).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes)
+{
+    return (uint64_t)((addr & 0x3ffffu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) |
+           ((uint64_t)(sbo_bytes >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+
+// Instruction descriptor for kind::f16 with bf16 inputs and fp32 accumulation: [4,6) D type
+// (1 = f32), [7,10) A type (1 = bf16), [10,13) B type, bit 15 / 16 A / B major (1 = MN-major),
+// [17,23) N >> 3, [24,29) M >> 4.
+__host__ __device__ constexpr uint32_t instr_desc(int m, int n, int b_mn_major)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(n >> 3) << 17) |
+           ((uint32_t)(m >> 4) << 24);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+
+// ---------------------------------------------------------------------------------------
+// the kernel
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kTcThreads, 1)
+tc_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap kv_map,
+                 DecodeParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    TcControl *ctl = reinterpret_cast<TcControl *>(smem + kSmemCtl);
+    const uint32_t smem_base = smem_u32(smem);
+
+    const int head_groups = (p.heads + kTcHeads - 1) / kTcHeads;
+    const int hg = blockIdx.x % head_groups;
+    const int s = (blockIdx.x / head_groups) % p.splits;
+    const int b = blockIdx.x / (head_groups * p.splits);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int h0 = hg * kTcHeads;
+
+    int n = __ldg(p.sel_len + b);
+    bool bad_len = false;
+    if (n < 0 || n > p.max_sel) {
+        bad_len = true;
+        n = 0;
+    }
+    int begin, end;
+    split_range(n, p.splits, s, begin, end);
+    const int tiles = (end - begin + kTile - 1) / kTile;
+
+    if (tiles == 0) {
+        // empty split: zero output / -inf log-sum-exp, no tensor-core work
+        if (threadIdx.x == 0 && bad_len) flag_status(p.status, OMNI_DEV_BAD_INDEX);
+        for (int r = warp; r < kTcHeads; r += kTcThreads / 32) {
+            const int h = h0 + r;
+            if (h >= p.heads) break;
+            if (p.splits == 1) {
+                uint4 *o = reinterpret_cast<uint4 *>(p.out + ((size_t)b * p.heads + h) * kDv);
+                for (int i = lane; i < kDv * 2 / 16; i += 32) o[i] = make_uint4(0, 0, 0, 0);
+                if (lane == 0) p.lse[(size_t)b * p.heads + h] = -INFINITY;
+            } else {
+                const size_t u = ((size_t)b * p.splits + s) * p.heads + h;
+                float4 *o = reinterpret_cast<float4 *>(p.part_out + u * kDv);
+                for (int i = lane; i < kDv / 4; i += 32) o[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (lane == 0) p.part_lse[u] = -INFINITY;
+            }
+        }
+        return;
+    }
+
+    // ---- set-up: barriers, tensor memory ------------------------------------------------
+    if (threadIdx.x == 0) {
+        mbar_init(&ctl->q_full, 1);
+        for (int i = 0; i < kStages; ++i) {
+            mbar_init(&ctl->kv_full[i], 1);
+            mbar_init(&ctl->kv_empty[i], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&ctl->s_full[i], 1);
+            mbar_init(&ctl->s_empty[i], 128);
+        }
+        mbar_init(&ctl->p_full, 128);
+        mbar_init(&ctl->pv_done, 1);
+        ctl->abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)),
+                     "r"(kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = ctl->tmem_base;
+    volatile uint32_t *abort_flag = &ctl->abort;
+
+    if (warp == 0) {
+        // =========================== producer ===========================================
+        const int32_t *sel = p.sel_idx + (size_t)b * p.max_sel;
+        const int32_t *pt = p.page_table + (size_t)b * p.max_pages;
+        if (lane == 0) {
+            mbar_expect_tx(&ctl->q_full, kTileBytes);
+            for (int c = 0; c < kPanels; ++c)
+                tma_box2d(smem_base + kSmemQ + c * kPanelBytes, &q_map, &ctl->q_full, c * 64, b * p.heads + h0);
+        }
+        bool any_bad = bad_len;
+        // rows of the tile after the current one are resolved while this one is in flight
+        auto resolve = [&](int tile, int &row_lo, int &row_hi, uint64_t &mask) {
+            const int j0 = begin + tile * kTile + lane, j1 = j0 + 32;
+            int64_t r0 = -1, r1 = -1;
+            if (j0 < end) {
+                r0 = resolve_row(pt, __ldg(sel + j0), p.max_pages, p.num_pages);
+                any_bad |= (r0 < 0);
+            }
+            if (j1 < end) {
+                r1 = resolve_row(pt, __ldg(sel + j1), p.max_pages, p.num_pages);
+                any_bad |= (r1 < 0);
+            }
+            const uint32_t m0 = __ballot_sync(0xffffffffu, r0 >= 0), m1 = __ballot_sync(0xffffffffu, r1 >= 0);
+            mask = (uint64_t)m0 | ((uint64_t)m1 << 32);
+            row_lo = r0 >= 0 ? (int)r0 : 0;      // masked tokens still load a real row (row 0)
+            row_hi = r1 >= 0 ? (int)r1 : 0;
+        };
+        int row_lo, row_hi;
+        uint64_t mask;
+        resolve(0, row_lo, row_hi, mask);
+        int issued = 0;
+        for (int i = 0; i < tiles; ++i) {
+            const int st = i % kStages;
+            int nrow_lo = 0, nrow_hi = 0;
+            uint64_t nmask = 0;
+            if (i + 1 < tiles) resolve(i + 1, nrow_lo, nrow_hi, nmask);
+            bool ok = true;
+            if (i >= kStages) ok = mbar_wait(&ctl->kv_empty[st], ((i / kStages) - 1) & 1);
+            ok = __all_sync(0xffffffffu, ok) && (*abort_flag == 0);
+            if (!ok) {
+                if (lane == 0) {
+                    flag_status(p.status, OMNI_DEV_TIMEOUT);
+                    *abort_flag = 1;
+                }
+                break;
+            }
+            // lane g < 16 gathers tokens 4g..4g+3 of the tile into rows 4g..4g+3 of every panel
+            int r[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int src = (4 * lane + k) & 31;
+                const int a = __shfl_sync(0xffffffffu, row_lo, src), c = __shfl_sync(0xffffffffu, row_hi, src);
+                r[k] = lane < 8 ? a : c;
+            }
+            if (lane == 0) {
+                ctl->valid_mask[st] = mask;
+                mbar_expect_tx(&ctl->kv_full[st], kTileBytes);
+            }
+            __syncwarp();
+            if (lane < 16) {
+                const uint32_t dst = smem_base + kSmemKV + st * kTileBytes + lane * 512;
+#pragma unroll
+                for (int c = 0; c < kPanels; ++c)
+                    tma_gather4(dst + c * kPanelBytes, &kv_map, &ctl->kv_full[st], c * 64, r[0], r[1], r[2], r[3]);
+            }
+            issued = i + 1;
+            row_lo = nrow_lo;
+            row_hi = nrow_hi;
+            mask = nmask;
+        }
+        if (__any_sync(0xffffffffu, any_bad) && lane == 0) flag_status(p.status, OMNI_DEV_BAD_INDEX);
+        if (*abort_flag) {
+            // let every copy this warp started land before the CTA can exit
+            for (int i = max(0, issued - kStages); i < issued; ++i) mbar_wait(&ctl->kv_full[i % kStages], (i / kStages) & 1);
+            mbar_wait(&ctl->q_full, 0);
+        }
+    } else if (warp == 1) {
+        // =========================== MMA issuer =========================================
+        if (lane == 0) {
+            constexpr uint32_t idesc_qk = instr_desc(kTcHeads, 32, 0);
+            constexpr uint32_t idesc_pv = instr_desc(kTcHeads, 256, 1);
+            const uint32_t q_addr = smem_base + kSmemQ, p_addr = smem_base + kSmemP;
+            bool ok = mbar_wait(&ctl->q_full, 0);
+            auto issue_qk = [&](int tile) {
+                const int st = tile % kStages, buf = tile & 1;
+                const uint32_t kv_addr = smem_base + kSmemKV + st * kTileBytes;
+                const uint32_t d = tmem + kColS + 32 * buf;
+#pragma unroll 4
+                for (int kk = 0; kk < kDqk / 16; ++kk) {
+                    const uint32_t off = (kk >> 2) * kPanelBytes + (kk & 3) * 32;
+                    const uint64_t a = smem_desc(q_addr + off, 16, 1024);
+                    tc_mma(d, a, smem_desc(kv_addr + off, 16, 1024), idesc_qk, kk > 0);
+                    tc_mma(d + kLane16, a, smem_desc(kv_addr + off + 32 * 128, 16, 1024), idesc_qk, kk > 0);
+                }
+                tc_commit(&ctl->s_full[buf]);
+            };
+            if (ok) ok = mbar_wait(&ctl->kv_full[0], 0);
+            if (ok) {
+                tc_fence_after();
+                issue_qk(0);
+            }
+            for (int i = 0; ok && i < tiles; ++i) {
+                if (i + 1 < tiles) {
+                    const int t = i + 1;
+                    ok = mbar_wait(&ctl->kv_full[t % kStages], (t / kStages) & 1);
+                    if (ok && t >= 2) ok = mbar_wait(&ctl->s_empty[t & 1], ((t >> 1) - 1) & 1);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_qk(t);
+                }
+                ok = mbar_wait(&ctl->p_full, i & 1);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t v_addr = smem_base + kSmemKV + (i % kStages) * kTileBytes;
+#pragma unroll
+                for (int k = 0; k < kTile / 16; ++k) {
+                    const uint64_t a = smem_desc(p_addr + k * 32, 16, 1024);
+                    const uint32_t acc = (i > 0 || k > 0) ? 1u : 0u;
+                    // V is the same tile read N-major: 64-column panels 8192 B apart, 8-token groups 1024 B apart
+                    tc_mma(tmem + kColO, a, smem_desc(v_addr + k * 2048, kPanelBytes, 1024), idesc_pv, acc);
+                    tc_mma(tmem + kColO + kLane16, a, smem_desc(v_addr + 4 * kPanelBytes + k * 2048, kPanelBytes, 1024),
+                           idesc_pv, acc);
+                }
+                tc_commit(&ctl->kv_empty[i % kStages]);
+                tc_commit(&ctl->pv_done);
+            }
+            if (!ok || *abort_flag) {
+                flag_status(p.status, OMNI_DEV_TIMEOUT);
+                *abort_flag = 1;
+            }
+        }
+        __syncwarp();
+    } else {
+        // =========================== softmax + epilogue =================================
+        const int quarter = warp & 3;                       // tensor-memory lane quarter of this warp
+        const int row = quarter * 16 + (lane & 15);         // head row within the CTA
+        const int half = lane >> 4;                         // token half of S / column half of O
+        const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+        uint8_t *p_row = smem + kSmemP + row * 128;
+        float m_ref = -INFINITY, l = 0.f;
+        bool ok = true;
+        for (int i = 0; i < tiles; ++i) {
+            const int buf = i & 1;
+            ok = mbar_wait(&ctl->s_full[buf], (i >> 1) & 1);
+            if (!__all_sync(0xffffffffu, ok)) {
+                ok = false;
+                break;
+            }
+            tc_fence_after();
+            uint32_t sv[32];
+            tc_ld32(tmem + lane_base + kColS + 32 * buf, sv);
+            tc_wait_ld();
+            tc_fence_before();
+            mbar_arrive(&ctl->s_empty[buf]);
+            const uint64_t vm = ctl->valid_mask[i % kStages];
+            const uint32_t valid = (uint32_t)(vm >> (32 * half));
+            float x[32];
+            float mt = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                x[j] = ((valid >> j) & 1u) ? __uint_as_float(sv[j]) * p.scale_log2 : -INFINITY;
+                mt = fmaxf(mt, x[j]);
+            }
+            mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, 16));
+            // move the reference only when the tile maximum leaves the window above it
+            float factor = 1.f;
+            bool moved = false;
+            if (mt > m_ref + kRescaleThreshold || (m_ref == -INFINITY && mt > -INFINITY)) {
+                factor = exp2f(m_ref - mt);                 // 0 on the first finite maximum
+                m_ref = mt;
+                moved = true;
+            }
+            const float mr = (m_ref == -INFINITY) ? 0.f : m_ref;
+            float sum = 0.f;
+            uint32_t pk[16];
+#pragma unroll
+            for (int j = 0; j < 32; j += 2) {
+                const float e0 = exp2f(x[j] - mr), e1 = exp2f(x[j + 1] - mr);
+                sum += e0 + e1;
+                pk[j >> 1] = pack_bf16(e0, e1);
+            }
+            l = l * factor + sum;
+            // P and O may only be touched once the previous tile's P V has finished
+            if (i > 0) {
+                ok = mbar_wait(&ctl->pv_done, (i - 1) & 1);
+                if (!__all_sync(0xffffffffu, ok)) {
+                    ok = false;
+                    break;
+                }
+                tc_fence_after();
+                if (__any_sync(0xffffffffu, moved)) {
+#pragma unroll 1
+                    for (int c = 0; c < 256; c += 32) {
+                        uint32_t ov[32];
+                        tc_ld32(tmem + lane_base + kColO + c, ov);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * factor);
+                        tc_st32(tmem + lane_base + kColO + c, ov);
+                    }
+                    tc_wait_st();
+                }
+            }
+            // P row: 64 tokens x bf16 = 128 B = eight 16-byte chunks, chunk c stored at c ^ (row % 8)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const int chunk = (half * 4 + c) ^ (row & 7);
+                *reinterpret_cast<uint4 *>(p_row + chunk * 16) =
+                    make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+            }
+            fence_async_smem();
+            tc_fence_before();
+            mbar_arrive(&ctl->p_full);
+        }
+        if (ok) {
+            ok = mbar_wait(&ctl->pv_done, (tiles - 1) & 1);
+            ok = __all_sync(0xffffffffu, ok);
+        }
+        if (ok) {
+            tc_fence_after();
+            const float lt = l + __shfl_xor_sync(0xffffffffu, l, 16);
+            const float inv = lt > 0.f ? 1.f / lt : 0.f;
+            const int h = h0 + row;
+            const bool store = h < p.heads;
+            const size_t u = p.splits == 1 ? ((size_t)b * p.heads + h) : (((size_t)b * p.splits + s) * p.heads + h);
+#pragma unroll 1
+            for (int c = 0; c < 256; c += 32) {
+                uint32_t ov[32];
+                __syncwarp();
+                tc_ld32(tmem + lane_base + kColO + c, ov);
+                tc_wait_ld();
+                const int col = half * 256 + c;
+                if (!store) {
+                    // padded head row: nothing to write
+                } else if (p.splits == 1) {
+                    uint4 *o = reinterpret_cast<uint4 *>(p.out + u * kDv + col);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        uint4 w;
+                        w.x = pack_bf16(__uint_as_float(ov[8 * j]) * inv, __uint_as_float(ov[8 * j + 1]) * inv);
+                        w.y = pack_bf16(__uint_as_float(ov[8 * j + 2]) * inv, __uint_as_float(ov[8 * j + 3]) * inv);
+                        w.z = pack_bf16(__uint_as_float(ov[8 * j + 4]) * inv, __uint_as_float(ov[8 * j + 5]) * inv);
+                        w.w = pack_bf16(__uint_as_float(ov[8 * j + 6]) * inv, __uint_as_float(ov[8 * j + 7]) * inv);
+                        o[j] = w;
+                    }
+                } else {
+                    float4 *o = reinterpret_cast<float4 *>(p.part_out + u * kDv + col);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        o[j] = make_float4(__uint_as_float(ov[4 * j]) * inv, __uint_as_float(ov[4 * j + 1]) * inv,
+                                           __uint_as_float(ov[4 * j + 2]) * inv, __uint_as_float(ov[4 * j + 3]) * inv);
+                }
+            }
+            if (store && half == 0) {
+                const float lse = lt > 0.f ? (m_ref + log2f(lt)) * kLn2 : -INFINITY;
+                if (p.splits == 1)
+                    p.lse[u] = lse;
+                else
+                    p.part_lse[u] = lse;
+            }
+        } else if (lane == 0) {
+            flag_status(p.status, OMNI_DEV_TIMEOUT);
+            *abort_flag = 1;
+        }
+    }
+
+    // ---- tear-down ----------------------------------------------------------------------
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// host side: tensor maps and launch
+// ---------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = [] {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess)
+            ptr = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(ptr);
+    }();
+    return fn;
+}
+
+// 2-D bf16 row-major [rows, 576] tensor, boxes of 64 columns x box_rows rows, 128-byte swizzle.
+inline bool make_row_map(CUtensorMap *map, const void *base, uint64_t rows, uint32_t box_rows)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)kDqk, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)kDqk * 2};
+    const cuuint32_t box[2] = {64, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+inline omni_status_t launch_tc_decode(const DecodeParams &p, cudaStream_t stream)
+{
+    static bool attr_set[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return OMNI_ERR_CUDA;
+    if (!attr_set[dev]) {
+        if (cudaFuncSetAttribute(tc_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBytes) !=
+            cudaSuccess)
+            return OMNI_ERR_CUDA;
+        attr_set[dev] = true;
+    }
+    CUtensorMap q_map, kv_map;
+    if (!make_row_map(&q_map, p.q, (uint64_t)p.batch * p.heads, kTcHeads)) return OMNI_ERR_CUDA;
+    if (!make_row_map(&kv_map, p.kv, (uint64_t)p.num_pages * kPage, 1)) return OMNI_ERR_CUDA;
+    const int head_groups = (p.heads + kTcHeads - 1) / kTcHeads;
+    const unsigned grid = (unsigned)(p.batch * p.splits * head_groups);
+    tc_decode_kernel<<<grid, kTcThreads, kTcSmemBytes, stream>>>(q_map, kv_map, p);
+    return cudaPeekAtLastError() == cudaSuccess ? OMNI_OK : OMNI_ERR_CUDA;
+}
+
+}  // namespace omni
