@@ -179,6 +179,42 @@ omni_status_t omni_sparse_mla_decode_host(const omni_mla_desc_t *desc, const voi
                                           int32_t *device_status, void *stream);
 
 /*
+ * Decode without a caller-supplied workspace (the paper has no counterpart: this is a
+ * packaging variant of omni_sparse_mla_decode, same arithmetic, same results).
+ *
+ * Who it is for: code that runs the decode step but may not allocate device memory, e.g. an
+ * attention plug-in inside a serving engine that has already handed every free byte of the
+ * GPU to its KV-cache pool, or a latency-critical decode loop where cudaMalloc / cudaFree are
+ * ruled out because they synchronise the device.  Such callers cannot provide the split-KV
+ * workspace, so here the library brings its own: a fixed array of OMNI_STATIC_SCRATCH_BYTES
+ * that is part of the library image.  The call itself performs no cudaMalloc, cudaFree or any
+ * other allocating call.
+ *
+ * Costs and rules that follow from that:
+ *   - every GPU on which the library is used keeps OMNI_STATIC_SCRATCH_BYTES (32 MiB) of
+ *     device memory occupied until the process exits;
+ *   - a problem whose omni_sparse_mla_workspace_bytes(desc) exceeds OMNI_STATIC_SCRATCH_BYTES
+ *     is rejected with OMNI_ERR_WORKSPACE and nothing is launched (lower desc->num_splits or
+ *     the batch, or use omni_sparse_mla_decode with a workspace of your own);
+ *   - the first call on each device looks up the array's device address (one runtime query,
+ *     with that device current) and caches it; make that first call during start-up, before
+ *     any stream capture begins;
+ *   - all calls on one device share the one array, which keeps whatever the previous call left
+ *     in it.  Nothing in it needs clearing (each call overwrites every partial result it
+ *     reads back), but two calls that overlap on the GPU, e.g. on different streams, race on
+ *     it: serialise them, or give the concurrent ones omni_sparse_mla_decode with separate
+ *     workspaces.
+ * All other arguments, results, alignment rules and status codes are those of
+ * omni_sparse_mla_decode.
+ */
+#define OMNI_STATIC_SCRATCH_BYTES (32u * 1024u * 1024u)
+omni_status_t omni_sparse_mla_decode_static(const omni_mla_desc_t *desc, const void *q,
+                                            const void *kv_cache, const int32_t *page_table,
+                                            const int32_t *sel_idx, const int32_t *sel_len,
+                                            void *out, float *lse, int32_t *device_status,
+                                            void *stream);
+
+/*
  * Profiling aid (no counterpart in the paper): when both events are non-NULL, every later
  * omni_sparse_mla_decode call on this thread's process records `before` and `after`
  * (cudaEvent_t passed as void*) on its stream immediately around the main decode kernel,

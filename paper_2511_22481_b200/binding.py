@@ -27,7 +27,7 @@ EXPORTS = (
     "omni_sparse_mla_workspace_bytes", "omni_sparse_mla_decode", "omni_sparse_mla_combine",
     "omni_sparse_mla_validate", "omni_sparse_mla_resolve_rows",
     "omni_sparse_mla_host_staging_bytes", "omni_sparse_mla_decode_host",
-    "omni_sparse_mla_set_profile_events",
+    "omni_sparse_mla_set_profile_events", "omni_sparse_mla_decode_static",
 )
 
 
@@ -87,6 +87,8 @@ def load() -> ctypes.CDLL:
     lib.omni_sparse_mla_host_staging_bytes.argtypes = [dp]
     lib.omni_sparse_mla_decode_host.restype = ctypes.c_int
     lib.omni_sparse_mla_decode_host.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp, sz, vp, vp]
+    lib.omni_sparse_mla_decode_static.restype = ctypes.c_int
+    lib.omni_sparse_mla_decode_static.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.omni_sparse_mla_set_profile_events.restype = None
     lib.omni_sparse_mla_set_profile_events.argtypes = [vp, vp]
     _lib = lib
@@ -161,6 +163,24 @@ def omni_sparse_mla_decode(desc, q, kv_cache, page_table, sel_idx, sel_len, out,
         None if workspace is None else ctypes.c_void_p(workspace.data_ptr()), ws_bytes,
         _ptr(device_status, torch.int32, "cuda", "device_status"), _stream(stream))
     _check(code, "omni_sparse_mla_decode")
+
+
+OMNI_STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
+
+
+def omni_sparse_mla_decode_static(desc, q, kv_cache, page_table, sel_idx, sel_len, out, lse,
+                                  device_status=None, stream=None) -> None:
+    """Decode for callers that may not allocate: no workspace argument, the split-KV scratch is
+    a fixed 32 MiB array inside the library (shared by all calls on a device, so calls that
+    overlap on the GPU race).  Raises OmniError(OMNI_ERR_WORKSPACE) if the problem needs more."""
+    code = load().omni_sparse_mla_decode_static(
+        ctypes.byref(desc), _ptr(q, torch.bfloat16, "cuda", "q"),
+        _ptr(kv_cache, torch.bfloat16, "cuda", "kv_cache"),
+        _ptr(page_table, torch.int32, "cuda", "page_table"),
+        _ptr(sel_idx, torch.int32, "cuda", "sel_idx"), _ptr(sel_len, torch.int32, "cuda", "sel_len"),
+        _ptr(out, torch.bfloat16, "cuda", "out"), _ptr(lse, torch.float32, "cuda", "lse"),
+        _ptr(device_status, torch.int32, "cuda", "device_status"), _stream(stream))
+    _check(code, "omni_sparse_mla_decode_static")
 
 
 def omni_sparse_mla_combine(desc, max_splits, part_out, part_lse, num_splits, out, lse,

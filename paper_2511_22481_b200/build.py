@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libomni_mla.so")
-SOURCES = [os.path.join(CSRC, "api.cu")]
+SOURCES = [os.path.join(CSRC, "api.cu"), os.path.join(CSRC, "static_scratch.cu")]
 
 
 def _deps():
