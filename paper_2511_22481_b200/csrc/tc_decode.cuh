@@ -3,8 +3,10 @@
 //
 // One CTA owns 64 heads of one (request, split) and walks the split's selected tokens in
 // 64-token tiles:
-//   warp 0      producer: resolves token positions to pool rows and gathers the rows with
-//               TMA (4 rows per instruction) into a 2-stage ring of 128B-swizzled tiles
+//   warp 0      producer: resolves token positions to pool rows and brings the rows into a
+//               2-stage ring of 128B-swizzled tiles with TMA: one 64x64 box per column panel
+//               when the tile is 64 consecutive pool rows (a page in order), otherwise
+//               row gathers of 4 rows per instruction
 //   warp 1      MMA issuer: S = Q K^T (M=64 heads, N=64 tokens, K=576) and O += P V
 //               (M=64, N=512, K=64); owns the tensor-memory allocation
 //   warps 2-5   softmax: read S from tensor memory, keep the running reference maximum and
@@ -14,10 +16,10 @@
 // Tensor-memory map (an M=64 accumulator occupies lanes 0-15 of each 32-lane quarter, so two
 // accumulators share a column range at lane offsets 0 and 16):
 //   columns   0..255  O   (lane offset 0: value columns 0..255, lane offset 16: 256..511)
-//   columns 256..287  S buffer 0 (lane offset 0: tokens 0..31 of the tile, 16: tokens 32..63)
-//   columns 288..319  S buffer 1
-// so every softmax thread owns half a row: lane l of a warp serves head row 16*(warp%4)+l%16
-// and the token / value-column half l/16.
+//   columns 256..319  S buffer 0 (one M=64 x N=64 accumulator, lanes 0-15 of each quarter)
+//   columns 320..383  S buffer 1
+// Every softmax thread owns half a row: lane l of a warp serves head row 16*(warp%4)+l%16 and
+// the token half (of S) / value-column half (of O) l/16.
 #pragma once
 
 #include <cuda.h>
@@ -200,9 +202,52 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 // ---------------------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------------------
+__device__ __forceinline__ bool mbar_test(uint64_t *bar, uint32_t parity)
+{
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return done != 0;
+}
+
+// MMA with the accumulate flag known at compile time (no predicate set-up per instruction).
+template <bool kAccumulate>
+__device__ __forceinline__ void tc_mma_c(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "n"(kAccumulate ? 1 : 0)
+        : "memory");
+}
+
+// 16 lanes x 32 columns twice: threads 0-15 of the warp read columns [c, c+32) of lanes 0-15 of
+// their quarter, threads 16-31 read columns [c+32, c+64) of the same lanes.  This is how the 64
+// rows of an M=64 accumulator (which live in lanes 0-15 of each quarter) are spread over all 32
+// threads of the warp that serves the quarter.
+__device__ __forceinline__ void tc_ld16x2(uint32_t taddr, uint32_t (&v)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.16x32bx2.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32], 32;"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr)
+        : "memory");
+}
+
 __global__ void __launch_bounds__(kTcThreads, 1)
 tc_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap kv_map,
-                 DecodeParams p)
+                 const __grid_constant__ CUtensorMap kv_page_map, DecodeParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -284,32 +329,41 @@ tc_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constan
                 tma_box2d(smem_base + kSmemQ + c * kPanelBytes, &q_map, &ctl->q_full, c * 64, b * p.heads + h0);
         }
         bool any_bad = bad_len;
-        // rows of the tile after the current one are resolved while this one is in flight
-        auto resolve = [&](int tile, int &row_lo, int &row_hi, uint64_t &mask) {
+        // Lane l serves tokens l and l+32 of a tile.  Token positions are fetched two tiles
+        // ahead and turned into pool rows one tile ahead, so neither dependent load sits
+        // between a freed stage and the copy that refills it.
+        auto fetch = [&](int tile, int &t0, int &t1) {
+            const int j0 = begin + tile * kTile + lane, j1 = j0 + 32;
+            t0 = (tile < tiles && j0 < end) ? __ldg(sel + j0) : 0;
+            t1 = (tile < tiles && j1 < end) ? __ldg(sel + j1) : 0;
+        };
+        auto lookup = [&](int tile, int t0, int t1, int &row_lo, int &row_hi, uint64_t &mask, bool &contig) {
             const int j0 = begin + tile * kTile + lane, j1 = j0 + 32;
             int64_t r0 = -1, r1 = -1;
             if (j0 < end) {
-                r0 = resolve_row(pt, __ldg(sel + j0), p.max_pages, p.num_pages);
+                r0 = resolve_row(pt, t0, p.max_pages, p.num_pages);
                 any_bad |= (r0 < 0);
             }
             if (j1 < end) {
-                r1 = resolve_row(pt, __ldg(sel + j1), p.max_pages, p.num_pages);
+                r1 = resolve_row(pt, t1, p.max_pages, p.num_pages);
                 any_bad |= (r1 < 0);
             }
             const uint32_t m0 = __ballot_sync(0xffffffffu, r0 >= 0), m1 = __ballot_sync(0xffffffffu, r1 >= 0);
             mask = (uint64_t)m0 | ((uint64_t)m1 << 32);
             row_lo = r0 >= 0 ? (int)r0 : 0;      // masked tokens still load a real row (row 0)
             row_hi = r1 >= 0 ? (int)r1 : 0;
+            const int base = __shfl_sync(0xffffffffu, row_lo, 0);
+            contig = __all_sync(0xffffffffu, r0 == (int64_t)base + lane && r1 == (int64_t)base + 32 + lane);
         };
-        int row_lo, row_hi;
+        int row_lo, row_hi, t0n, t1n;
         uint64_t mask;
-        resolve(0, row_lo, row_hi, mask);
+        bool contig;
+        fetch(0, t0n, t1n);
+        lookup(0, t0n, t1n, row_lo, row_hi, mask, contig);
+        fetch(1, t0n, t1n);
         int issued = 0;
         for (int i = 0; i < tiles; ++i) {
             const int st = i % kStages;
-            int nrow_lo = 0, nrow_hi = 0;
-            uint64_t nmask = 0;
-            if (i + 1 < tiles) resolve(i + 1, nrow_lo, nrow_hi, nmask);
             bool ok = true;
             if (i >= kStages) ok = mbar_wait(&ctl->kv_empty[st], ((i / kStages) - 1) & 1);
             ok = __all_sync(0xffffffffu, ok) && (*abort_flag == 0);
@@ -320,29 +374,35 @@ tc_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constan
                 }
                 break;
             }
-            // lane g < 16 gathers tokens 4g..4g+3 of the tile into rows 4g..4g+3 of every panel
-            int r[4];
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const int src = (4 * lane + k) & 31;
-                const int a = __shfl_sync(0xffffffffu, row_lo, src), c = __shfl_sync(0xffffffffu, row_hi, src);
-                r[k] = lane < 8 ? a : c;
-            }
             if (lane == 0) {
                 ctl->valid_mask[st] = mask;
                 mbar_expect_tx(&ctl->kv_full[st], kTileBytes);
             }
             __syncwarp();
-            if (lane < 16) {
-                const uint32_t dst = smem_base + kSmemKV + st * kTileBytes + lane * 512;
+            const uint32_t stage = smem_base + kSmemKV + st * kTileBytes;
+            if (contig) {
+                // 64 consecutive pool rows (a whole page in order): one 64x64 box per column panel
+                if (lane < kPanels)
+                    tma_box2d(stage + lane * kPanelBytes, &kv_page_map, &ctl->kv_full[st], lane * 64, row_lo - lane);
+            } else {
+                // scattered rows: lane g < 16 gathers tokens 4g..4g+3 into rows 4g..4g+3 of every panel
+                int r[4];
 #pragma unroll
-                for (int c = 0; c < kPanels; ++c)
-                    tma_gather4(dst + c * kPanelBytes, &kv_map, &ctl->kv_full[st], c * 64, r[0], r[1], r[2], r[3]);
+                for (int k = 0; k < 4; ++k) {
+                    const int src = (4 * lane + k) & 31;
+                    const int a = __shfl_sync(0xffffffffu, row_lo, src), c = __shfl_sync(0xffffffffu, row_hi, src);
+                    r[k] = lane < 8 ? a : c;
+                }
+                if (lane < 16) {
+#pragma unroll
+                    for (int c = 0; c < kPanels; ++c)
+                        tma_gather4(stage + lane * 512 + c * kPanelBytes, &kv_map, &ctl->kv_full[st], c * 64, r[0], r[1],
+                                    r[2], r[3]);
+                }
             }
             issued = i + 1;
-            row_lo = nrow_lo;
-            row_hi = nrow_hi;
-            mask = nmask;
+            if (i + 1 < tiles) lookup(i + 1, t0n, t1n, row_lo, row_hi, mask, contig);
+            fetch(i + 2, t0n, t1n);
         }
         if (__any_sync(0xffffffffu, any_bad) && lane == 0) flag_status(p.status, OMNI_DEV_BAD_INDEX);
         if (*abort_flag) {
@@ -353,54 +413,69 @@ tc_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constan
     } else if (warp == 1) {
         // =========================== MMA issuer =========================================
         if (lane == 0) {
-            constexpr uint32_t idesc_qk = instr_desc(kTcHeads, 32, 0);
+            constexpr uint32_t idesc_qk = instr_desc(kTcHeads, kTile, 0);
             constexpr uint32_t idesc_pv = instr_desc(kTcHeads, 256, 1);
-            const uint32_t q_addr = smem_base + kSmemQ, p_addr = smem_base + kSmemP;
+            const uint64_t q_desc = smem_desc(smem_base + kSmemQ, 16, 1024);
+            const uint64_t p_desc = smem_desc(smem_base + kSmemP, 16, 1024);
             bool ok = mbar_wait(&ctl->q_full, 0);
-            auto issue_qk = [&](int tile) {
-                const int st = tile % kStages, buf = tile & 1;
-                const uint32_t kv_addr = smem_base + kSmemKV + st * kTileBytes;
-                const uint32_t d = tmem + kColS + 32 * buf;
-#pragma unroll 4
-                for (int kk = 0; kk < kDqk / 16; ++kk) {
-                    const uint32_t off = (kk >> 2) * kPanelBytes + (kk & 3) * 32;
-                    const uint64_t a = smem_desc(q_addr + off, 16, 1024);
-                    tc_mma(d, a, smem_desc(kv_addr + off, 16, 1024), idesc_qk, kk > 0);
-                    tc_mma(d + kLane16, a, smem_desc(kv_addr + off + 32 * 128, 16, 1024), idesc_qk, kk > 0);
-                }
-                tc_commit(&ctl->s_full[buf]);
-            };
-            if (ok) ok = mbar_wait(&ctl->kv_full[0], 0);
-            if (ok) {
-                tc_fence_after();
-                issue_qk(0);
-            }
-            for (int i = 0; ok && i < tiles; ++i) {
-                if (i + 1 < tiles) {
-                    const int t = i + 1;
-                    ok = mbar_wait(&ctl->kv_full[t % kStages], (t / kStages) & 1);
-                    if (ok && t >= 2) ok = mbar_wait(&ctl->s_empty[t & 1], ((t >> 1) - 1) & 1);
-                    if (!ok) break;
-                    tc_fence_after();
-                    issue_qk(t);
-                }
-                ok = mbar_wait(&ctl->p_full, i & 1);
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t v_addr = smem_base + kSmemKV + (i % kStages) * kTileBytes;
+            // S(t) = Q K(t)^T : 36 k-steps of 16 columns; panel c of Q against panel c of the stage
+            auto issue_qk = [&](int t) {
+                const uint64_t k_desc = smem_desc(smem_base + kSmemKV + (t % kStages) * kTileBytes, 16, 1024);
+                const uint32_t d = tmem + kColS + 64 * (t & 1);
+                tc_mma_c<false>(d, q_desc, k_desc, idesc_qk);
 #pragma unroll
-                for (int k = 0; k < kTile / 16; ++k) {
-                    const uint64_t a = smem_desc(p_addr + k * 32, 16, 1024);
-                    const uint32_t acc = (i > 0 || k > 0) ? 1u : 0u;
-                    // V is the same tile read N-major: 64-column panels 8192 B apart, 8-token groups 1024 B apart
-                    tc_mma(tmem + kColO, a, smem_desc(v_addr + k * 2048, kPanelBytes, 1024), idesc_pv, acc);
-                    tc_mma(tmem + kColO + kLane16, a, smem_desc(v_addr + 4 * kPanelBytes + k * 2048, kPanelBytes, 1024),
-                           idesc_pv, acc);
+                for (int kk = 1; kk < kDqk / 16; ++kk) {
+                    const uint32_t off = ((kk >> 2) * kPanelBytes + (kk & 3) * 32) >> 4;
+                    tc_mma_c<true>(d, q_desc + off, k_desc + off, idesc_qk);
+                }
+                tc_commit(&ctl->s_full[t & 1]);
+            };
+            // O += P(i) V(i) : the stage read N-major (64-column panels 8192 B apart, 8-token groups
+            // 1024 B apart); value columns 0..255 and 256..511 go to the two interleaved accumulators
+            auto issue_pv = [&](int i) {
+                const uint64_t v_desc = smem_desc(smem_base + kSmemKV + (i % kStages) * kTileBytes, kPanelBytes, 1024);
+                if (i == 0) {
+                    tc_mma_c<false>(tmem + kColO, p_desc, v_desc, idesc_pv);
+                    tc_mma_c<false>(tmem + kColO + kLane16, p_desc, v_desc + ((4 * kPanelBytes) >> 4), idesc_pv);
+                } else {
+                    tc_mma_c<true>(tmem + kColO, p_desc, v_desc, idesc_pv);
+                    tc_mma_c<true>(tmem + kColO + kLane16, p_desc, v_desc + ((4 * kPanelBytes) >> 4), idesc_pv);
+                }
+#pragma unroll
+                for (int k = 1; k < kTile / 16; ++k) {
+                    tc_mma_c<true>(tmem + kColO, p_desc + ((k * 32) >> 4), v_desc + ((k * 2048) >> 4), idesc_pv);
+                    tc_mma_c<true>(tmem + kColO + kLane16, p_desc + ((k * 32) >> 4),
+                                   v_desc + ((4 * kPanelBytes + k * 2048) >> 4), idesc_pv);
                 }
                 tc_commit(&ctl->kv_empty[i % kStages]);
                 tc_commit(&ctl->pv_done);
+            };
+            // Issue whichever of "next Q K^T" and "next P V" has its inputs ready, so a late tile
+            // never holds back the P V that frees a stage.
+            int next_qk = 0, next_pv = 0;
+            long long idle_since = clock64();
+            while (ok && next_pv < tiles) {
+                bool progress = false;
+                if (next_qk < tiles && next_qk <= next_pv + 1 &&
+                    mbar_test(&ctl->kv_full[next_qk % kStages], (next_qk / kStages) & 1) &&
+                    (next_qk < 2 || mbar_test(&ctl->s_empty[next_qk & 1], ((next_qk >> 1) - 1) & 1))) {
+                    tc_fence_after();
+                    issue_qk(next_qk);
+                    ++next_qk;
+                    progress = true;
+                }
+                if (next_pv < next_qk && mbar_test(&ctl->p_full, next_pv & 1)) {
+                    tc_fence_after();
+                    issue_pv(next_pv);
+                    ++next_pv;
+                    progress = true;
+                }
+                if (progress)
+                    idle_since = clock64();
+                else if (clock64() - idle_since > kWaitCycles || *abort_flag)
+                    ok = false;
             }
-            if (!ok || *abort_flag) {
+            if (!ok) {
                 flag_status(p.status, OMNI_DEV_TIMEOUT);
                 *abort_flag = 1;
             }
@@ -424,7 +499,7 @@ tc_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constan
             }
             tc_fence_after();
             uint32_t sv[32];
-            tc_ld32(tmem + lane_base + kColS + 32 * buf, sv);
+            tc_ld16x2(tmem + lane_base + kColS + 64 * buf, sv);
             tc_wait_ld();
             tc_fence_before();
             mbar_arrive(&ctl->s_empty[buf]);
@@ -594,12 +669,13 @@ inline omni_status_t launch_tc_decode(const DecodeParams &p, cudaStream_t stream
             return OMNI_ERR_CUDA;
         attr_set[dev] = true;
     }
-    CUtensorMap q_map, kv_map;
+    CUtensorMap q_map, kv_map, kv_page_map;
     if (!make_row_map(&q_map, p.q, (uint64_t)p.batch * p.heads, kTcHeads)) return OMNI_ERR_CUDA;
     if (!make_row_map(&kv_map, p.kv, (uint64_t)p.num_pages * kPage, 1)) return OMNI_ERR_CUDA;
+    if (!make_row_map(&kv_page_map, p.kv, (uint64_t)p.num_pages * kPage, kTile)) return OMNI_ERR_CUDA;
     const int head_groups = (p.heads + kTcHeads - 1) / kTcHeads;
     const unsigned grid = (unsigned)(p.batch * p.splits * head_groups);
-    tc_decode_kernel<<<grid, kTcThreads, kTcSmemBytes, stream>>>(q_map, kv_map, p);
+    tc_decode_kernel<<<grid, kTcThreads, kTcSmemBytes, stream>>>(q_map, kv_map, kv_page_map, p);
     return cudaPeekAtLastError() == cudaSuccess ? OMNI_OK : OMNI_ERR_CUDA;
 }
 
