@@ -8,6 +8,7 @@
 #include "common.cuh"
 #include "simt_decode.cuh"
 #include "tc_decode.cuh"
+#include "tc2_decode.cuh"
 
 namespace omni {
 namespace {
@@ -55,11 +56,15 @@ bool desc_ok(const omni_mla_desc_t *d)
 
 bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
-// Work units (CTAs) one split of one request occupies in the kernel that will run.
+// More than 64 heads run on the paired-CTA kernel (one cluster of two CTAs per work unit).
+bool use_pair_kernel(const omni_mla_desc_t *d) { return !(d->flags & OMNI_FLAG_SIMT) && d->num_heads > kTcHeads; }
+
+// Work units one split of one request occupies in the kernel that will run.
 int units_per_request(const omni_mla_desc_t *d)
 {
     if (d->flags & OMNI_FLAG_SIMT)
         return (d->num_heads + kSimtWarps * kSimtHeadsPerWarp - 1) / (kSimtWarps * kSimtHeadsPerWarp);
+    if (use_pair_kernel(d)) return 1;
     return (d->num_heads + kTcHeads - 1) / kTcHeads;
 }
 
@@ -70,8 +75,10 @@ int choose_splits(const omni_mla_desc_t *d, int sm_count)
 {
     if (d->num_splits >= 1) return d->num_splits;
     if (sm_count <= 0) sm_count = 148;
-    const int granules = (d->max_sel + kTile - 1) / kTile;
+    const int granule = use_pair_kernel(d) ? kC2Tile : kTile;
+    const int granules = (d->max_sel + granule - 1) / granule;
     const long units = (long)d->batch * units_per_request(d);
+    if (use_pair_kernel(d)) sm_count /= 2;               // a work unit occupies two SMs
     long best_cost = -1;
     int best = 1;
     for (int s = 1; s <= kMaxSplits && s <= granules; ++s) {
@@ -217,7 +224,7 @@ omni_status_t omni_sparse_mla_decode(const omni_mla_desc_t *desc, const void *q,
         simt_decode_kernel<<<grid, kSimtWarps * 32, 0, stream>>>(p);
         if (cudaPeekAtLastError() != cudaSuccess) return OMNI_ERR_CUDA;
     } else {
-        omni_status_t st = launch_tc_decode(p, stream);
+        omni_status_t st = use_pair_kernel(desc) ? launch_tc2_decode(p, stream) : launch_tc_decode(p, stream);
         if (st != OMNI_OK) return st;
     }
     if (g_profile_before && g_profile_after) cudaEventRecord(g_profile_after, stream);

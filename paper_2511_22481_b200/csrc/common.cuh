@@ -34,13 +34,15 @@ struct DecodeParams {
 };
 
 // Token range [begin, end) of split s of a request with n selected tokens: the n tokens are
-// cut into 64-token granules and the granules are dealt out in contiguous, equal runs.
-__device__ __forceinline__ void split_range(int n, int splits, int s, int &begin, int &end)
+// cut into granules (64 tokens unless a kernel works on larger tiles) and the granules are
+// dealt out in contiguous, equal runs.
+__device__ __forceinline__ void split_range(int n, int splits, int s, int &begin, int &end,
+                                            int granule = kTile)
 {
-    const int granules = (n + kTile - 1) / kTile;
+    const int granules = (n + granule - 1) / granule;
     const int per = (granules + splits - 1) / splits;
-    begin = min(n, s * per * kTile);
-    end = min(n, (s + 1) * per * kTile);
+    begin = min(n, s * per * granule);
+    end = min(n, (s + 1) * per * granule);
 }
 
 // Logical token position -> physical pool row, or -1 if the entry breaks the index contract.
