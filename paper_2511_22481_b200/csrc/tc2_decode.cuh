@@ -14,9 +14,11 @@
 // byte leaves HBM once when the pair runs together).
 //
 // Shared memory has room for one tile per role, so the buffers are refilled piecewise while
-// they are consumed: the 9 column panels of the K role each have their own full/empty barrier
-// pair (a panel is reloaded for the next tile as soon as its four MMAs retire) and the V role
-// is split in its two 64-token halves.  All MMAs are issued by one thread of CTA 0 in
+// they are consumed: the 9 column panels of the K role form three groups with their own
+// full/empty barrier pairs (a group is reloaded for the next tile as soon as its twelve MMAs
+// retire) and the V role is split in its two 64-token halves.  Every refill is ONE 3-D TMA box
+// {64 columns, 64 rows, 3 or 4 panels}: the copy engine sustains only about 4 M instructions/s
+// per SM, so 8 KiB boxes cap an SM near 32 GB/s while 24-72 KiB boxes reach 90-150 GB/s.  All MMAs are issued by one thread of CTA 0 in
 // "whatever is ready" order; completion is broadcast to both CTAs with multicast commits.
 //
 // Warps per CTA: 0 K-role producer, 1 MMA issuer (CTA 0 only) + tensor-memory owner,
@@ -46,11 +48,13 @@ constexpr int kC2SmemCtlBytes = 2048;
 constexpr int kC2SmemBytes = kC2SmemCtl + kC2SmemCtlBytes + 1024;
 constexpr uint32_t kC2ColS = 256;
 constexpr int kMaskRing = 4;
+constexpr int kKGroups = 3;                           // the K role is refilled in 3 groups of 3 column panels
+constexpr int kKGroupBytes = 3 * kPanelBytes;
 
 struct C2Control {
     uint64_t q_full;
-    uint64_t k_full[kPanels];
-    uint64_t k_empty[kPanels];
+    uint64_t k_full[kKGroups];
+    uint64_t k_empty[kKGroups];
     uint64_t v_full[2];
     uint64_t v_empty[2];
     uint64_t s_full[2];
@@ -83,7 +87,9 @@ __device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, uint32_t rank)
 
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
 {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+    // default (CTA-scope release) semantics: a cluster-scope release costs ~0.6 us per arrive here,
+    // and what must be ordered before it is already ordered by the tcgen05 / async-proxy fences
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 
 __device__ __forceinline__ void cluster_sync_all()
@@ -100,6 +106,18 @@ __device__ __forceinline__ void tma_box2d_pair(uint32_t dst, const CUtensorMap *
         "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
         " [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(map), "r"(col), "r"(row), "r"(bar_cluster_addr)
+        : "memory");
+}
+
+// 3-D box {64 columns, 64 rows, n column panels}: lands panel-major, i.e. as n consecutive
+// [64 rows x 128 B] swizzled panels, in one instruction.
+__device__ __forceinline__ void tma_box3d_pair(uint32_t dst, const CUtensorMap *map, uint32_t bar_cluster_addr,
+                                               int row, int panel)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(map), "r"(0), "r"(row), "r"(panel), "r"(bar_cluster_addr)
         : "memory");
 }
 
@@ -124,6 +142,34 @@ __device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t a_desc, ui
         : "memory");
 }
 
+// The same, executed by a whole converged warp: one elected lane issues the instruction.  The
+// descriptors arrive as 32-bit halves so that stepping through a tile is a 32-bit add.
+template <bool kAccumulate>
+__device__ __forceinline__ void tc_mma_pair_elect(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo,
+                                                  uint32_t b_hi, uint32_t idesc)
+{
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t.reg .b64 da, db;\n\t"
+        "mov.b64 da, {%1, %2};\n\t"
+        "mov.b64 db, {%3, %4};\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "elect.sync _|q, 0xffffffff;\n\t"
+        "@q tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %5, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "n"(kAccumulate ? 1 : 0)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_commit_pair_elect(uint64_t *bar)
+{
+    const uint16_t both = 3;
+    asm volatile(
+        "{\n\t.reg .pred q;\n\t"
+        "elect.sync _|q, 0xffffffff;\n\t"
+        "@q tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;\n\t}"
+        ::"r"(smem_u32(bar)), "h"(both)
+        : "memory");
+}
+
 // Arrive on the barrier at this shared-memory offset in BOTH CTAs once all MMAs issued so far
 // by this thread have retired.
 __device__ __forceinline__ void tc_commit_pair(uint64_t *bar)
@@ -137,7 +183,8 @@ __device__ __forceinline__ void tc_commit_pair(uint64_t *bar)
 
 __global__ void __launch_bounds__(kC2Threads, 1)
 tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap kv_map,
-                  const __grid_constant__ CUtensorMap kv_page_map, DecodeParams p)
+                  const __grid_constant__ CUtensorMap kv_k_map, const __grid_constant__ CUtensorMap kv_v_map,
+                  DecodeParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -148,7 +195,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     const int pair = blockIdx.x >> 1;
     const int s = pair % p.splits;
     const int b = pair / p.splits;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;  // warp-uniform
     const int h0 = (int)rank * kTcHeads;
 
     int n = __ldg(p.sel_len + b);
@@ -184,7 +231,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     // ---- set-up ---------------------------------------------------------------------------
     if (threadIdx.x == 0) {
         mbar_init(&ctl->q_full, 1);
-        for (int i = 0; i < kPanels; ++i) {
+        for (int i = 0; i < kKGroups; ++i) {
             mbar_init(&ctl->k_full[i], 1);
             mbar_init(&ctl->k_empty[i], 1);
         }
@@ -216,30 +263,34 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     const int32_t *sel = p.sel_idx + (size_t)b * p.max_sel;
     const int32_t *pt = p.page_table + (size_t)b * p.max_pages;
 
-    // Rows of one 64-token half of a tile: lane l serves tokens l and l+32 of the half.
-    auto fetch_half = [&](int tile, int half, int &t0, int &t1) {
-        const int j0 = begin + tile * kC2Tile + half * 64 + lane, j1 = j0 + 32;
-        t0 = (tile < tiles && j0 < end) ? __ldg(sel + j0) : 0;
-        t1 = (tile < tiles && j1 < end) ? __ldg(sel + j1) : 0;
+    // Index pipeline of the producers.  Lane l serves tokens l and l+32 of one 64-token half of a
+    // tile.  The three dependent steps (token position -> page id -> pool row) run in different
+    // loop iterations, one tile apart, so no load is consumed in the iteration that issued it.
+    struct HalfIdx {
+        int t0, t1;        // token positions (stage 1)
+        int pg0, pg1;      // physical page ids, -1 if the position breaks the contract (stage 2)
     };
-    auto lookup_half = [&](int tile, int half, int t0, int t1, int &row_lo, int &row_hi, uint64_t &mask, bool &contig,
-                           bool &any_bad) {
+    auto stage_tokens = [&](int tile, int half, HalfIdx &x) {
         const int j0 = begin + tile * kC2Tile + half * 64 + lane, j1 = j0 + 32;
-        int64_t r0 = -1, r1 = -1;
-        if (j0 < end) {
-            r0 = resolve_row(pt, t0, p.max_pages, p.num_pages);
-            any_bad |= (r0 < 0);
-        }
-        if (j1 < end) {
-            r1 = resolve_row(pt, t1, p.max_pages, p.num_pages);
-            any_bad |= (r1 < 0);
-        }
+        x.t0 = (tile < tiles && j0 < end) ? __ldg(sel + j0) : -1;
+        x.t1 = (tile < tiles && j1 < end) ? __ldg(sel + j1) : -1;
+    };
+    auto stage_pages = [&](HalfIdx &x) {
+        x.pg0 = (x.t0 >= 0 && x.t0 / kPage < p.max_pages) ? __ldg(pt + x.t0 / kPage) : -1;
+        x.pg1 = (x.t1 >= 0 && x.t1 / kPage < p.max_pages) ? __ldg(pt + x.t1 / kPage) : -1;
+    };
+    auto stage_rows = [&](int tile, int half, const HalfIdx &x, int &row_lo, int &row_hi, uint64_t &mask, bool &contig,
+                          bool &any_bad) {
+        const int j0 = begin + tile * kC2Tile + half * 64 + lane, j1 = j0 + 32;
+        const bool ok0 = x.pg0 >= 0 && (int64_t)x.pg0 < p.num_pages, ok1 = x.pg1 >= 0 && (int64_t)x.pg1 < p.num_pages;
+        any_bad |= (j0 < end && !ok0) || (j1 < end && !ok1);
+        const int r0 = ok0 ? x.pg0 * kPage + x.t0 % kPage : -1, r1 = ok1 ? x.pg1 * kPage + x.t1 % kPage : -1;
         const uint32_t m0 = __ballot_sync(0xffffffffu, r0 >= 0), m1 = __ballot_sync(0xffffffffu, r1 >= 0);
         mask = (uint64_t)m0 | ((uint64_t)m1 << 32);
-        row_lo = r0 >= 0 ? (int)r0 : 0;
-        row_hi = r1 >= 0 ? (int)r1 : 0;
+        row_lo = r0 >= 0 ? r0 : 0;           // masked tokens still load a real row (row 0)
+        row_hi = r1 >= 0 ? r1 : 0;
         const int base = __shfl_sync(0xffffffffu, row_lo, 0);
-        contig = __all_sync(0xffffffffu, r0 == (int64_t)base + lane && r1 == (int64_t)base + 32 + lane);
+        contig = __all_sync(0xffffffffu, r0 == base + lane && r1 == base + 32 + lane);
     };
     // Lane g < 16 takes the rows of tokens 4g..4g+3 of a half.
     auto rows_of_four = [&](int row_lo, int row_hi, int (&r)[4]) {
@@ -256,22 +307,28 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         const uint32_t q_bar = map_to_rank(smem_u32(&ctl->q_full), 0);
         if (lane == 0) {
             if (rank == 0) mbar_expect_tx(&ctl->q_full, 2 * kTileBytes);
-            for (int c = 0; c < kPanels; ++c)
-                tma_box2d_pair(smem_base + kC2SmemQ + c * kPanelBytes, &q_map, q_bar, c * 64, b * p.heads + h0);
+            tma_box3d_pair(smem_base + kC2SmemQ, &q_map, q_bar, b * p.heads + h0, 0);
         }
         bool any_bad = bad_len;
         // This CTA's K rows are the tokens of half `rank`; the other half is resolved too because
         // the softmax threads need the validity of all 128 tokens of a tile.
-        int own_lo, own_hi, oth_lo, oth_hi, t0a, t1a, t0b, t1b;
+        const int own = (int)rank, oth = own ^ 1;
+        HalfIdx a1, b1, a2, b2;              // own / other half, one and two tiles ahead
+        int own_lo, own_hi, oth_lo, oth_hi;
         uint64_t mask_own, mask_oth;
         bool contig, contig_oth;
-        const int own = (int)rank, oth = own ^ 1;
-        fetch_half(0, own, t0a, t1a);
-        fetch_half(0, oth, t0b, t1b);
-        lookup_half(0, own, t0a, t1a, own_lo, own_hi, mask_own, contig, any_bad);
-        lookup_half(0, oth, t0b, t1b, oth_lo, oth_hi, mask_oth, contig_oth, any_bad);
-        fetch_half(1, own, t0a, t1a);
-        fetch_half(1, oth, t0b, t1b);
+        stage_tokens(0, own, a1);
+        stage_tokens(0, oth, b1);
+        stage_pages(a1);
+        stage_pages(b1);
+        stage_rows(0, own, a1, own_lo, own_hi, mask_own, contig, any_bad);
+        stage_rows(0, oth, b1, oth_lo, oth_hi, mask_oth, contig_oth, any_bad);
+        stage_tokens(1, own, a1);
+        stage_tokens(1, oth, b1);
+        stage_pages(a1);
+        stage_pages(b1);
+        stage_tokens(2, own, a2);
+        stage_tokens(2, oth, b2);
         bool ok = true;
         for (int i = 0; ok && i < tiles; ++i) {
             if (lane == 0) {
@@ -281,27 +338,35 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
             }
             int r[4];
             rows_of_four(own_lo, own_hi, r);
-            for (int c = 0; c < kPanels; ++c) {
-                if (i > 0) ok = mbar_wait(&ctl->k_empty[c], (i - 1) & 1);
+            for (int g = 0; g < kKGroups; ++g) {
+                if (i > 0) ok = mbar_wait(&ctl->k_empty[g], (i - 1) & 1);
                 ok = __all_sync(0xffffffffu, ok) && (*abort_flag == 0);
                 if (!ok) break;
-                const uint32_t bar = map_to_rank(smem_u32(&ctl->k_full[c]), 0);
-                if (lane == 0 && rank == 0) mbar_expect_tx(&ctl->k_full[c], 2 * kPanelBytes);
+                const uint32_t bar = map_to_rank(smem_u32(&ctl->k_full[g]), 0);
+                if (lane == 0 && rank == 0) mbar_expect_tx(&ctl->k_full[g], 2 * kKGroupBytes);
                 __syncwarp();
-                const uint32_t dst = smem_base + kC2SmemK + c * kPanelBytes;
+                const uint32_t dst = smem_base + kC2SmemK + g * kKGroupBytes;
                 if (contig) {
-                    if (lane == 0) tma_box2d_pair(dst, &kv_page_map, bar, c * 64, own_lo);
+                    if (lane == 0) tma_box3d_pair(dst, &kv_k_map, bar, own_lo, 3 * g);
                 } else if (lane < 16) {
-                    tma_gather4_pair(dst + lane * 512, &kv_map, bar, c * 64, r[0], r[1], r[2], r[3]);
+#pragma unroll
+                    for (int c = 0; c < 3; ++c)
+                        tma_gather4_pair(dst + c * kPanelBytes + lane * 512, &kv_map, bar, (3 * g + c) * 64, r[0], r[1], r[2],
+                                         r[3]);
                 }
             }
             if (!ok) break;
+            // advance the index pipeline: rows of tile i+1, page ids of tile i+2, positions of tile i+3
             if (i + 1 < tiles) {
-                lookup_half(i + 1, own, t0a, t1a, own_lo, own_hi, mask_own, contig, any_bad);
-                lookup_half(i + 1, oth, t0b, t1b, oth_lo, oth_hi, mask_oth, contig_oth, any_bad);
+                stage_rows(i + 1, own, a1, own_lo, own_hi, mask_own, contig, any_bad);
+                stage_rows(i + 1, oth, b1, oth_lo, oth_hi, mask_oth, contig_oth, any_bad);
             }
-            fetch_half(i + 2, own, t0a, t1a);
-            fetch_half(i + 2, oth, t0b, t1b);
+            a1 = a2;
+            b1 = b2;
+            stage_pages(a1);
+            stage_pages(b1);
+            stage_tokens(i + 3, own, a2);
+            stage_tokens(i + 3, oth, b2);
         }
         if (!ok && lane == 0) {
             flag_status(p.status, OMNI_DEV_TIMEOUT);
@@ -311,14 +376,19 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     } else if (warp == 6) {
         // =========================== V-role producer =====================================
         bool any_bad = false;
-        int lo[2], hi[2], t0[2], t1[2];
+        HalfIdx x1[2], x2[2];
+        int lo[2], hi[2];
         uint64_t mask_unused;
         bool contig[2];
-        for (int h = 0; h < 2; ++h) fetch_half(0, h, t0[h], t1[h]);
-        for (int h = 0; h < 2; ++h) lookup_half(0, h, t0[h], t1[h], lo[h], hi[h], mask_unused, contig[h], any_bad);
-        for (int h = 0; h < 2; ++h) fetch_half(1, h, t0[h], t1[h]);
+        for (int h = 0; h < 2; ++h) {
+            stage_tokens(0, h, x1[h]);
+            stage_pages(x1[h]);
+            stage_rows(0, h, x1[h], lo[h], hi[h], mask_unused, contig[h], any_bad);
+            stage_tokens(1, h, x1[h]);
+            stage_pages(x1[h]);
+            stage_tokens(2, h, x2[h]);
+        }
         bool ok = true;
-        const int col0 = (int)rank * 256;
         for (int i = 0; ok && i < tiles; ++i) {
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
@@ -330,23 +400,26 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
                 __syncwarp();
                 const uint32_t dst = smem_base + kC2SmemV + h * kC2VHalfBytes;
                 if (contig[h]) {
-                    if (lane < 4) tma_box2d_pair(dst + lane * kPanelBytes, &kv_page_map, bar, col0 + lane * 64, lo[h] - lane);
+                    if (lane == 0) tma_box3d_pair(dst, &kv_v_map, bar, lo[h], 4 * (int)rank);
                 } else {
                     int r[4];
                     rows_of_four(lo[h], hi[h], r);
                     if (lane < 16) {
 #pragma unroll
                         for (int c = 0; c < 4; ++c)
-                            tma_gather4_pair(dst + c * kPanelBytes + lane * 512, &kv_map, bar, col0 + c * 64, r[0], r[1],
-                                             r[2], r[3]);
+                            tma_gather4_pair(dst + c * kPanelBytes + lane * 512, &kv_map, bar, ((int)rank * 4 + c) * 64, r[0],
+                                             r[1], r[2], r[3]);
                     }
                 }
             }
             if (!ok) break;
-            if (i + 1 < tiles)
-                for (int h = 0; h < 2; ++h)
-                    lookup_half(i + 1, h, t0[h], t1[h], lo[h], hi[h], mask_unused, contig[h], any_bad);
-            for (int h = 0; h < 2; ++h) fetch_half(i + 2, h, t0[h], t1[h]);
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                if (i + 1 < tiles) stage_rows(i + 1, h, x1[h], lo[h], hi[h], mask_unused, contig[h], any_bad);
+                x1[h] = x2[h];
+                stage_pages(x1[h]);
+                stage_tokens(i + 3, h, x2[h]);
+            }
         }
         if (!ok && lane == 0) {
             flag_status(p.status, OMNI_DEV_TIMEOUT);
@@ -354,13 +427,18 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         }
     } else if (warp == 1) {
         // =========================== MMA issuer (CTA 0 only) =============================
-        if (rank == 0 && lane == 0) {
+        // The whole warp runs this loop with warp-uniform control flow and one elected lane issues
+        // each MMA / commit: descriptor arithmetic then stays cheap enough to issue an MMA every
+        // 32 clocks, which a lone diverged thread cannot.
+        if (rank == 0) {
             constexpr uint32_t idesc_qk = instr_desc(128, kC2Tile, 0);
             constexpr uint32_t idesc_pv = instr_desc(128, 256, 1);
             const uint64_t q_desc = smem_desc(smem_base + kC2SmemQ, 16, 1024);
             const uint64_t k_desc = smem_desc(smem_base + kC2SmemK, 16, 1024);
             const uint64_t p_desc = smem_desc(smem_base + kC2SmemP, 16, 1024);
             const uint64_t v_desc = smem_desc(smem_base + kC2SmemV, kPanelBytes, 1024);
+            const uint32_t q_lo = (uint32_t)q_desc, k_lo = (uint32_t)k_desc, p_lo = (uint32_t)p_desc, v_lo = (uint32_t)v_desc;
+            const uint32_t kmaj_hi = (uint32_t)(q_desc >> 32), v_hi = (uint32_t)(v_desc >> 32);
             bool ok = mbar_wait(&ctl->q_full, 0);
             int qk_t = 0, qk_c = 0, pv_t = 0, pv_h = 0;
             long long idle_since = clock64();
@@ -370,22 +448,24 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
                 if (pv_t < qk_t && (pv_h == 1 || mbar_test(&ctl->p_full, pv_t & 1)) &&
                     mbar_test(&ctl->v_full[pv_h], pv_t & 1)) {
                     tc_fence_after();
-                    const uint64_t a = p_desc + ((pv_h * kPanelBytes) >> 4);
-                    const uint64_t bd = v_desc + ((pv_h * kC2VHalfBytes) >> 4);
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        const uint64_t ak = a + ((k * 32) >> 4), bk = bd + ((k * 2048) >> 4);
-                        if (pv_t == 0 && pv_h == 0 && k == 0) {
-                            tc_mma_pair<false>(tmem + kColO, ak, bk, idesc_pv);
-                            tc_mma_pair<false>(tmem + kColO + 128, ak, bk + ((2 * kPanelBytes) >> 4), idesc_pv);
-                        } else {
-                            tc_mma_pair<true>(tmem + kColO, ak, bk, idesc_pv);
-                            tc_mma_pair<true>(tmem + kColO + 128, ak, bk + ((2 * kPanelBytes) >> 4), idesc_pv);
-                        }
+                    const uint32_t a = p_lo + ((pv_h * kPanelBytes) >> 4);
+                    const uint32_t bd = v_lo + ((pv_h * kC2VHalfBytes) >> 4);
+                    if (pv_t == 0 && pv_h == 0) {
+                        tc_mma_pair_elect<false>(tmem + kColO, a, kmaj_hi, bd, v_hi, idesc_pv);
+                        tc_mma_pair_elect<false>(tmem + kColO + 128, a, kmaj_hi, bd + ((2 * kPanelBytes) >> 4), v_hi, idesc_pv);
+                    } else {
+                        tc_mma_pair_elect<true>(tmem + kColO, a, kmaj_hi, bd, v_hi, idesc_pv);
+                        tc_mma_pair_elect<true>(tmem + kColO + 128, a, kmaj_hi, bd + ((2 * kPanelBytes) >> 4), v_hi, idesc_pv);
                     }
-                    tc_commit_pair(&ctl->v_empty[pv_h]);
+#pragma unroll
+                    for (int k = 1; k < 4; ++k) {
+                        const uint32_t ak = a + ((k * 32) >> 4), bk = bd + ((k * 2048) >> 4);
+                        tc_mma_pair_elect<true>(tmem + kColO, ak, kmaj_hi, bk, v_hi, idesc_pv);
+                        tc_mma_pair_elect<true>(tmem + kColO + 128, ak, kmaj_hi, bk + ((2 * kPanelBytes) >> 4), v_hi, idesc_pv);
+                    }
+                    tc_commit_pair_elect(&ctl->v_empty[pv_h]);
                     if (pv_h == 1) {
-                        tc_commit_pair(&ctl->pv_done);
+                        tc_commit_pair_elect(&ctl->pv_done);
                         ++pv_t;
                         pv_h = 0;
                     } else {
@@ -393,22 +473,24 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
                     }
                     progress = true;
                 }
-                // ---- one 64-column panel of S = Q K^T ----
+                // ---- one group of three 64-column panels of S = Q K^T ----
                 if (qk_t < tiles && mbar_test(&ctl->k_full[qk_c], qk_t & 1) &&
                     (qk_c > 0 || qk_t < 2 || mbar_test(&ctl->s_empty[qk_t & 1], ((qk_t >> 1) - 1) & 1))) {
                     tc_fence_after();
                     const uint32_t d = tmem + kC2ColS + 64 * (qk_t & 1);
-                    const uint32_t off = (qk_c * kPanelBytes) >> 4;
+                    const uint32_t off = (qk_c * kKGroupBytes) >> 4;
                     if (qk_c == 0)
-                        tc_mma_pair<false>(d, q_desc, k_desc, idesc_qk);
+                        tc_mma_pair_elect<false>(d, q_lo, kmaj_hi, k_lo, kmaj_hi, idesc_qk);
                     else
-                        tc_mma_pair<true>(d, q_desc + off, k_desc + off, idesc_qk);
+                        tc_mma_pair_elect<true>(d, q_lo + off, kmaj_hi, k_lo + off, kmaj_hi, idesc_qk);
 #pragma unroll
-                    for (int k = 1; k < 4; ++k)
-                        tc_mma_pair<true>(d, q_desc + off + ((k * 32) >> 4), k_desc + off + ((k * 32) >> 4), idesc_qk);
-                    tc_commit_pair(&ctl->k_empty[qk_c]);
-                    if (++qk_c == kPanels) {
-                        tc_commit_pair(&ctl->s_full[qk_t & 1]);
+                    for (int k = 1; k < 12; ++k) {
+                        const uint32_t o = off + (((k >> 2) * kPanelBytes + (k & 3) * 32) >> 4);
+                        tc_mma_pair_elect<true>(d, q_lo + o, kmaj_hi, k_lo + o, kmaj_hi, idesc_qk);
+                    }
+                    tc_commit_pair_elect(&ctl->k_empty[qk_c]);
+                    if (++qk_c == kKGroups) {
+                        tc_commit_pair_elect(&ctl->s_full[qk_t & 1]);
                         qk_c = 0;
                         ++qk_t;
                     }
@@ -418,8 +500,9 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
                     idle_since = clock64();
                 else if (clock64() - idle_since > kWaitCycles || *abort_flag)
                     ok = false;
+                ok = __all_sync(0xffffffffu, ok);
             }
-            if (!ok) {
+            if (!ok && lane == 0) {
                 flag_status(p.status, OMNI_DEV_TIMEOUT);
                 *abort_flag = 1;
             }
@@ -602,10 +685,11 @@ inline omni_status_t launch_tc2_decode(const DecodeParams &p, cudaStream_t strea
             return OMNI_ERR_CUDA;
         attr_set[dev] = true;
     }
-    CUtensorMap q_map, kv_map, kv_page_map;
-    if (!make_row_map(&q_map, p.q, (uint64_t)p.batch * p.heads, kTcHeads)) return OMNI_ERR_CUDA;
+    CUtensorMap q_map, kv_map, kv_k_map, kv_v_map;
+    if (!make_panel_map(&q_map, p.q, (uint64_t)p.batch * p.heads, kPanels)) return OMNI_ERR_CUDA;
     if (!make_row_map(&kv_map, p.kv, (uint64_t)p.num_pages * kPage, 1)) return OMNI_ERR_CUDA;
-    if (!make_row_map(&kv_page_map, p.kv, (uint64_t)p.num_pages * kPage, kTile)) return OMNI_ERR_CUDA;
+    if (!make_panel_map(&kv_k_map, p.kv, (uint64_t)p.num_pages * kPage, 3)) return OMNI_ERR_CUDA;
+    if (!make_panel_map(&kv_v_map, p.kv, (uint64_t)p.num_pages * kPage, 4)) return OMNI_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(p.batch * p.splits * 2));
     cfg.blockDim = dim3(kC2Threads);
@@ -618,7 +702,7 @@ inline omni_status_t launch_tc2_decode(const DecodeParams &p, cudaStream_t strea
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, tc2_decode_kernel, q_map, kv_map, kv_page_map, p) == cudaSuccess ? OMNI_OK
+    return cudaLaunchKernelEx(&cfg, tc2_decode_kernel, q_map, kv_map, kv_k_map, kv_v_map, p) == cudaSuccess ? OMNI_OK
                                                                                                       : OMNI_ERR_CUDA;
 }
 

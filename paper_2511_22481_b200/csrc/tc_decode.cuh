@@ -658,6 +658,22 @@ inline bool make_row_map(CUtensorMap *map, const void *base, uint64_t rows, uint
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The same tensor seen as [rows, 9 panels of 64 columns]: 3-D boxes {64 columns, 64 rows, n panels}
+// land in shared memory panel by panel ([64 rows x 128 B] each, 128-byte swizzle), which is the
+// operand layout of the MMAs, so one instruction fills up to a whole 72 KiB tile.
+inline bool make_panel_map(CUtensorMap *map, const void *base, uint64_t rows, uint32_t box_panels)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[3] = {64, (cuuint64_t)rows, (cuuint64_t)kPanels};
+    const cuuint64_t strides[2] = {(cuuint64_t)kDqk * 2, 128};
+    const cuuint32_t box[3] = {64, (cuuint32_t)kTile, box_panels};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 inline omni_status_t launch_tc_decode(const DecodeParams &p, cudaStream_t stream)
 {
     static bool attr_set[64] = {};
