@@ -109,6 +109,13 @@ omni_status_t launch_combine(int batch, int heads, int max_splits, const float *
                              const float *part_lse, const int32_t *num_splits, void *out,
                              float *lse, cudaStream_t stream)
 {
+    // Keep the shared-memory / L1 split the decode kernel needs: alternating between two splits
+    // makes every launch wait for the SMs to be reconfigured.
+    static bool carveout_set = false;
+    if (!carveout_set) {
+        cudaFuncSetAttribute(combine_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
+        carveout_set = true;
+    }
     combine_kernel<<<batch * heads, 128, 0, stream>>>(part_out, part_lse, num_splits, max_splits,
                                                       heads, static_cast<__nv_bfloat16 *>(out), lse);
     return cudaPeekAtLastError() == cudaSuccess ? OMNI_OK : OMNI_ERR_CUDA;

@@ -3,66 +3,74 @@
 // A cluster of two CTAs owns all heads of one (request, split): CTA r serves heads
 // [64r, 64r+64).  The pair issues cta_group::2 MMAs with M = 128 (64 rows per CTA), which run
 // the tensor pipe of each SM at full rate where a lone M = 64 MMA runs it at half rate, and it
-// halves the operand bytes each SM must hold:
-//   S = Q K^T   M=128, N=128 tokens, K=576: every CTA supplies its 64 Q rows and the K rows of
-//               ITS 64 tokens of the 128-token tile ("K role": 64 tokens x 576 columns)
-//   O += P V    M=128, N=256 per instruction, K=128 tokens: every CTA supplies its 64 P rows
-//               and, for all 128 tokens, ITS 256 value columns ("V role": 128 tokens x 256
-//               columns; CTA r holds columns [256r, 256r+256))
+// halves the operand bytes each SM must hold.  Per 64-token tile:
+//   S = Q K^T   M=128, N=64 tokens, K=576: every CTA supplies its 64 Q rows and the K rows of
+//               ITS 32 tokens of the tile ("K role": 32 tokens x 576 columns, 36 KiB)
+//   O += P V    M=128, N=256 per instruction (two of them), K=64 tokens: every CTA supplies its
+//               64 P rows and, for all 64 tokens, ITS 256 value columns ("V role": 64 tokens x
+//               256 columns, 32 KiB; CTA r holds columns [256r, 256r+256))
 // The two roles overlap only in a quarter of the tile, at different addresses in the two CTAs,
-// so each role is loaded on its own (1.9x the tile's bytes cross L2 -> shared memory, but each
-// byte leaves HBM once when the pair runs together).
+// so each role is loaded on its own (1.9x the tile's bytes cross L2 -> shared memory, which L2
+// sustains; each byte leaves HBM once because the pair runs together).
 //
-// Shared memory has room for one tile per role, so the buffers are refilled piecewise while
-// they are consumed: the 9 column panels of the K role form three groups with their own
-// full/empty barrier pairs (a group is reloaded for the next tile as soon as its twelve MMAs
-// retire) and the V role is split in its two 64-token halves.  Every refill is ONE 3-D TMA box
-// {64 columns, 64 rows, 3 or 4 panels}: the copy engine sustains only about 4 M instructions/s
-// per SM, so 8 KiB boxes cap an SM near 32 GB/s while 24-72 KiB boxes reach 90-150 GB/s.  All MMAs are issued by one thread of CTA 0 in
-// "whatever is ready" order; completion is broadcast to both CTAs with multicast commits.
+// Both roles, P and S are double buffered, so the loads of tile i+2 are in flight while tile i
+// is consumed and Q K^T of tile i+1 overlaps the softmax of tile i.  Every refill is ONE 3-D TMA
+// box {64 columns, rows, panels}: the copy engine sustains only about 4 M instructions/s per SM,
+// so 8 KiB boxes cap an SM near 32 GB/s while 32-72 KiB boxes reach 90-150 GB/s.  Tiles that are
+// not 64 consecutive pool rows fall back to 4-row gathers.
+//
+// All MMAs are issued by warp 1 of CTA 0 in "whatever is ready" order: the whole warp runs the
+// loop with warp-uniform control flow and one elected lane issues each instruction (a lone
+// diverged thread cannot feed the tensor pipe: it needs ~110 clocks per MMA, the elected form
+// issues one every 25-64 clocks).  Completion is broadcast to both CTAs with multicast commits.
 //
 // Warps per CTA: 0 K-role producer, 1 MMA issuer (CTA 0 only) + tensor-memory owner,
-// 2-5 softmax / epilogue, 6 V-role producer.
+// 2-5 softmax / epilogue, 6 V-role producer, 7 L2 prefetcher (CTA 0 only): shared memory holds
+// only two tiles, about one HBM latency of work, so whole pages are pulled into L2 a few tiles
+// ahead and the shared-memory refills then hit L2.
 //
 // Tensor memory per CTA (a 64-row slice of an M=128 pair accumulator keeps columns [0, N/2) in
 // lanes 0-63 and columns [N/2, N) in lanes 64-127):
 //   columns   0..255  O: two N=256 accumulators; lane L, column x  <->  head row L%64,
 //                        value column 256*(L/64) + x
-//   columns 256..319  S buffer 0: lane L, column x <-> head row L%64, token 64*(L/64) + x
-//   columns 320..383  S buffer 1
+//   columns 256..287  S buffer 0: lane L, column x <-> head row L%64, token 32*(L/64) + x
+//   columns 288..319  S buffer 1
 #pragma once
+
+#include <type_traits>
 
 #include "tc_decode.cuh"
 
 namespace omni {
 
-constexpr int kC2Tile = 128;                          // tokens per tile of the pair
-constexpr int kC2Threads = 224;
-constexpr int kC2SmemQ = 0;                           // 9 panels x 8 KiB
-constexpr int kC2SmemK = kC2SmemQ + kTileBytes;       // K role: 9 panels x [64 tokens x 128 B]
-constexpr int kC2VHalfBytes = 4 * kPanelBytes;        // V role, one 64-token half: 4 panels
-constexpr int kC2SmemV = kC2SmemK + kTileBytes;
-constexpr int kC2SmemP = kC2SmemV + 2 * kC2VHalfBytes;  // P: 2 panels x [64 heads x 128 B]
+constexpr int kC2Tile = 64;                              // tokens per tile of the pair
+constexpr int kC2Threads = 256;
+constexpr int kPrefetchAhead = 5;                         // tiles the L2 prefetch runs ahead of Q K^T
+constexpr int kC2KBytes = kPanels * 32 * 128;            // K role: 9 panels x [32 tokens x 128 B]
+constexpr int kC2KPanel = 32 * 128;
+constexpr int kC2VBytes = 4 * kPanelBytes;               // V role: 4 panels x [64 tokens x 128 B]
+constexpr int kC2SmemQ = 0;                              // 9 panels x [64 heads x 128 B]
+constexpr int kC2SmemK = kC2SmemQ + kTileBytes;          // 2 stages
+constexpr int kC2SmemV = kC2SmemK + 2 * kC2KBytes;       // 2 stages
+constexpr int kC2SmemP = kC2SmemV + 2 * kC2VBytes;       // 2 buffers x [64 heads x 128 B]
 constexpr int kC2SmemCtl = kC2SmemP + 2 * kPanelBytes;
 constexpr int kC2SmemCtlBytes = 2048;
 constexpr int kC2SmemBytes = kC2SmemCtl + kC2SmemCtlBytes + 1024;
 constexpr uint32_t kC2ColS = 256;
 constexpr int kMaskRing = 4;
-constexpr int kKGroups = 3;                           // the K role is refilled in 3 groups of 3 column panels
-constexpr int kKGroupBytes = 3 * kPanelBytes;
 
 struct C2Control {
     uint64_t q_full;
-    uint64_t k_full[kKGroups];
-    uint64_t k_empty[kKGroups];
+    uint64_t k_full[2];
+    uint64_t k_empty[2];
     uint64_t v_full[2];
-    uint64_t v_empty[2];
     uint64_t s_full[2];
     uint64_t s_empty[2];
-    uint64_t p_full;
-    uint64_t pv_done;
+    uint64_t p_full[2];
+    uint64_t pv_done[2];                 // P V of a tile retired: frees its V stage and its P buffer
     uint64_t x_bar;                      // softmax threads: row-maximum exchange
-    uint64_t valid_mask[kMaskRing][2];   // per tile: validity of tokens 0..63 and 64..127
+    uint64_t exit_bar;                   // both CTAs of the pair are done with tensor memory
+    uint64_t valid_mask[kMaskRing];      // per tile: validity of its 64 tokens
     float xchg[2][2][64];                // [tile parity][token half][head row]
     uint32_t tmem_base;
     uint32_t abort;
@@ -92,25 +100,22 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
     asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 
+// Execution-only rendezvous of the pair (no memory ordering): used before the tensor-memory
+// release, where the release-ordered form would first wait for every global store of the
+// epilogue to be acknowledged (about 9 us here).
+__device__ __forceinline__ void cluster_sync_relaxed()
+{
+    asm volatile("barrier.cluster.arrive.relaxed.aligned;\n\tbarrier.cluster.wait.aligned;" ::: "memory");
+}
+
 __device__ __forceinline__ void cluster_sync_all()
 {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
-// Box load of one CTA of a pair; the transaction bytes are credited to `bar_cluster_addr`, which
-// may be a barrier of the other CTA of the pair.
-__device__ __forceinline__ void tma_box2d_pair(uint32_t dst, const CUtensorMap *map, uint32_t bar_cluster_addr,
-                                               int col, int row)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
-        " [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(col), "r"(row), "r"(bar_cluster_addr)
-        : "memory");
-}
-
-// 3-D box {64 columns, 64 rows, n column panels}: lands panel-major, i.e. as n consecutive
-// [64 rows x 128 B] swizzled panels, in one instruction.
+// 3-D box {64 columns, box rows, n column panels} loaded by one CTA of a pair: lands panel-major,
+// i.e. as n consecutive [rows x 128 B] swizzled panels.  The transaction bytes are credited to
+// `bar_cluster_addr`, which may be a barrier of the other CTA of the pair.
 __device__ __forceinline__ void tma_box3d_pair(uint32_t dst, const CUtensorMap *map, uint32_t bar_cluster_addr,
                                                int row, int panel)
 {
@@ -131,18 +136,7 @@ __device__ __forceinline__ void tma_gather4_pair(uint32_t dst, const CUtensorMap
         : "memory");
 }
 
-template <bool kAccumulate>
-__device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "n"(kAccumulate ? 1 : 0)
-        : "memory");
-}
-
-// The same, executed by a whole converged warp: one elected lane issues the instruction.  The
+// Pair MMA executed by a whole converged warp: one elected lane issues the instruction.  The
 // descriptors arrive as 32-bit halves so that stepping through a tile is a 32-bit add.
 template <bool kAccumulate>
 __device__ __forceinline__ void tc_mma_pair_elect(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo,
@@ -159,6 +153,8 @@ __device__ __forceinline__ void tc_mma_pair_elect(uint32_t d_tmem, uint32_t a_lo
         : "memory");
 }
 
+// Arrive on the barrier at this shared-memory offset in BOTH CTAs once all MMAs issued so far by
+// the elected lane have retired.
 __device__ __forceinline__ void tc_commit_pair_elect(uint64_t *bar)
 {
     const uint16_t both = 3;
@@ -170,21 +166,10 @@ __device__ __forceinline__ void tc_commit_pair_elect(uint64_t *bar)
         : "memory");
 }
 
-// Arrive on the barrier at this shared-memory offset in BOTH CTAs once all MMAs issued so far
-// by this thread have retired.
-__device__ __forceinline__ void tc_commit_pair(uint64_t *bar)
-{
-    const uint16_t both = 3;
-    asm volatile(
-        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-        ::"r"(smem_u32(bar)), "h"(both)
-        : "memory");
-}
-
 __global__ void __launch_bounds__(kC2Threads, 1)
 tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap kv_map,
                   const __grid_constant__ CUtensorMap kv_k_map, const __grid_constant__ CUtensorMap kv_v_map,
-                  DecodeParams p)
+                  const __grid_constant__ CUtensorMap kv_tile_map, DecodeParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -231,19 +216,17 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     // ---- set-up ---------------------------------------------------------------------------
     if (threadIdx.x == 0) {
         mbar_init(&ctl->q_full, 1);
-        for (int i = 0; i < kKGroups; ++i) {
+        for (int i = 0; i < 2; ++i) {
             mbar_init(&ctl->k_full[i], 1);
             mbar_init(&ctl->k_empty[i], 1);
-        }
-        for (int i = 0; i < 2; ++i) {
             mbar_init(&ctl->v_full[i], 1);
-            mbar_init(&ctl->v_empty[i], 1);
             mbar_init(&ctl->s_full[i], 1);
             mbar_init(&ctl->s_empty[i], 8);      // one arrival per softmax warp of either CTA
+            mbar_init(&ctl->p_full[i], 8);
+            mbar_init(&ctl->pv_done[i], 1);
         }
-        mbar_init(&ctl->p_full, 8);
-        mbar_init(&ctl->pv_done, 1);
         mbar_init(&ctl->x_bar, 128);
+        mbar_init(&ctl->exit_bar, 2);
         ctl->abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -263,110 +246,92 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     const int32_t *sel = p.sel_idx + (size_t)b * p.max_sel;
     const int32_t *pt = p.page_table + (size_t)b * p.max_pages;
 
-    // Index pipeline of the producers.  Lane l serves tokens l and l+32 of one 64-token half of a
-    // tile.  The three dependent steps (token position -> page id -> pool row) run in different
-    // loop iterations, one tile apart, so no load is consumed in the iteration that issued it.
-    struct HalfIdx {
+    // Index pipeline of the producers.  Lane l serves tokens l and l+32 of a tile.  The three
+    // dependent steps (token position -> page id -> pool row) run in different loop iterations,
+    // one tile apart, so no load is consumed in the iteration that issued it.
+    struct TileIdx {
         int t0, t1;        // token positions (stage 1)
         int pg0, pg1;      // physical page ids, -1 if the position breaks the contract (stage 2)
     };
-    auto stage_tokens = [&](int tile, int half, HalfIdx &x) {
-        const int j0 = begin + tile * kC2Tile + half * 64 + lane, j1 = j0 + 32;
+    auto stage_tokens = [&](int tile, TileIdx &x) {
+        const int j0 = begin + tile * kC2Tile + lane, j1 = j0 + 32;
         x.t0 = (tile < tiles && j0 < end) ? __ldg(sel + j0) : -1;
         x.t1 = (tile < tiles && j1 < end) ? __ldg(sel + j1) : -1;
     };
-    auto stage_pages = [&](HalfIdx &x) {
+    auto stage_pages = [&](TileIdx &x) {
         x.pg0 = (x.t0 >= 0 && x.t0 / kPage < p.max_pages) ? __ldg(pt + x.t0 / kPage) : -1;
         x.pg1 = (x.t1 >= 0 && x.t1 / kPage < p.max_pages) ? __ldg(pt + x.t1 / kPage) : -1;
     };
-    auto stage_rows = [&](int tile, int half, const HalfIdx &x, int &row_lo, int &row_hi, uint64_t &mask, bool &contig,
-                          bool &any_bad) {
-        const int j0 = begin + tile * kC2Tile + half * 64 + lane, j1 = j0 + 32;
+    // row_lo / row_hi: pool rows of tokens lane and lane+32 (row 0 stands in for masked tokens);
+    // contig: all 64 tokens valid and in consecutive rows; contig_lo / contig_hi: the same per 32.
+    auto stage_rows = [&](int tile, const TileIdx &x, int &row_lo, int &row_hi, uint64_t &mask, bool &contig,
+                          bool &contig_lo, bool &contig_hi, bool &any_bad) {
+        const int j0 = begin + tile * kC2Tile + lane, j1 = j0 + 32;
         const bool ok0 = x.pg0 >= 0 && (int64_t)x.pg0 < p.num_pages, ok1 = x.pg1 >= 0 && (int64_t)x.pg1 < p.num_pages;
         any_bad |= (j0 < end && !ok0) || (j1 < end && !ok1);
         const int r0 = ok0 ? x.pg0 * kPage + x.t0 % kPage : -1, r1 = ok1 ? x.pg1 * kPage + x.t1 % kPage : -1;
         const uint32_t m0 = __ballot_sync(0xffffffffu, r0 >= 0), m1 = __ballot_sync(0xffffffffu, r1 >= 0);
         mask = (uint64_t)m0 | ((uint64_t)m1 << 32);
-        row_lo = r0 >= 0 ? r0 : 0;           // masked tokens still load a real row (row 0)
+        row_lo = r0 >= 0 ? r0 : 0;
         row_hi = r1 >= 0 ? r1 : 0;
-        const int base = __shfl_sync(0xffffffffu, row_lo, 0);
-        contig = __all_sync(0xffffffffu, r0 == base + lane && r1 == base + 32 + lane);
-    };
-    // Lane g < 16 takes the rows of tokens 4g..4g+3 of a half.
-    auto rows_of_four = [&](int row_lo, int row_hi, int (&r)[4]) {
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const int src = (4 * lane + k) & 31;
-            const int a = __shfl_sync(0xffffffffu, row_lo, src), c = __shfl_sync(0xffffffffu, row_hi, src);
-            r[k] = lane < 8 ? a : c;
-        }
+        const int base_lo = __shfl_sync(0xffffffffu, row_lo, 0), base_hi = __shfl_sync(0xffffffffu, row_hi, 0);
+        contig_lo = __all_sync(0xffffffffu, r0 == base_lo + lane);
+        contig_hi = __all_sync(0xffffffffu, r1 == base_hi + lane);
+        contig = contig_lo && contig_hi && base_hi == base_lo + 32;
     };
 
     if (warp == 0) {
         // =========================== K-role producer =====================================
+        // This CTA's K rows are tokens [32*rank, 32*rank+32) of every tile.
         const uint32_t q_bar = map_to_rank(smem_u32(&ctl->q_full), 0);
         if (lane == 0) {
             if (rank == 0) mbar_expect_tx(&ctl->q_full, 2 * kTileBytes);
             tma_box3d_pair(smem_base + kC2SmemQ, &q_map, q_bar, b * p.heads + h0, 0);
         }
         bool any_bad = bad_len;
-        // This CTA's K rows are the tokens of half `rank`; the other half is resolved too because
-        // the softmax threads need the validity of all 128 tokens of a tile.
-        const int own = (int)rank, oth = own ^ 1;
-        HalfIdx a1, b1, a2, b2;              // own / other half, one and two tiles ahead
-        int own_lo, own_hi, oth_lo, oth_hi;
-        uint64_t mask_own, mask_oth;
-        bool contig, contig_oth;
-        stage_tokens(0, own, a1);
-        stage_tokens(0, oth, b1);
-        stage_pages(a1);
-        stage_pages(b1);
-        stage_rows(0, own, a1, own_lo, own_hi, mask_own, contig, any_bad);
-        stage_rows(0, oth, b1, oth_lo, oth_hi, mask_oth, contig_oth, any_bad);
-        stage_tokens(1, own, a1);
-        stage_tokens(1, oth, b1);
-        stage_pages(a1);
-        stage_pages(b1);
-        stage_tokens(2, own, a2);
-        stage_tokens(2, oth, b2);
+        TileIdx x1, x2;                      // one and two tiles ahead
+        int row_lo, row_hi;
+        uint64_t mask;
+        bool contig, contig_lo, contig_hi;
+        stage_tokens(0, x1);
+        stage_pages(x1);
+        stage_rows(0, x1, row_lo, row_hi, mask, contig, contig_lo, contig_hi, any_bad);
+        stage_tokens(1, x1);
+        stage_pages(x1);
+        stage_tokens(2, x2);
         bool ok = true;
         for (int i = 0; ok && i < tiles; ++i) {
+            const int st = i & 1;
             if (lane == 0) {
-                ctl->valid_mask[i % kMaskRing][own] = mask_own;
-                ctl->valid_mask[i % kMaskRing][oth] = mask_oth;
+                ctl->valid_mask[i % kMaskRing] = mask;
                 __threadfence_block();
             }
-            int r[4];
-            rows_of_four(own_lo, own_hi, r);
-            for (int g = 0; g < kKGroups; ++g) {
-                if (i > 0) ok = mbar_wait(&ctl->k_empty[g], (i - 1) & 1);
-                ok = __all_sync(0xffffffffu, ok) && (*abort_flag == 0);
-                if (!ok) break;
-                const uint32_t bar = map_to_rank(smem_u32(&ctl->k_full[g]), 0);
-                if (lane == 0 && rank == 0) mbar_expect_tx(&ctl->k_full[g], 2 * kKGroupBytes);
-                __syncwarp();
-                const uint32_t dst = smem_base + kC2SmemK + g * kKGroupBytes;
-                if (contig) {
-                    if (lane == 0) tma_box3d_pair(dst, &kv_k_map, bar, own_lo, 3 * g);
-                } else if (lane < 16) {
+            if (i >= 2) ok = mbar_wait(&ctl->k_empty[st], ((i >> 1) - 1) & 1);
+            ok = __all_sync(0xffffffffu, ok) && (*abort_flag == 0);
+            if (!ok) break;
+            const uint32_t bar = map_to_rank(smem_u32(&ctl->k_full[st]), 0);
+            if (lane == 0 && rank == 0) mbar_expect_tx(&ctl->k_full[st], 2 * kC2KBytes);
+            __syncwarp();
+            const uint32_t dst = smem_base + kC2SmemK + st * kC2KBytes;
+            const int own_row = rank ? row_hi : row_lo;
+            if (rank ? contig_hi : contig_lo) {
+                if (lane == 0) tma_box3d_pair(dst, &kv_k_map, bar, own_row, 0);
+            } else {
+                // lane g < 8 gathers tokens 4g..4g+3 of this CTA's 32 into rows 4g..4g+3 of every panel
+                int r[4];
 #pragma unroll
-                    for (int c = 0; c < 3; ++c)
-                        tma_gather4_pair(dst + c * kPanelBytes + lane * 512, &kv_map, bar, (3 * g + c) * 64, r[0], r[1], r[2],
-                                         r[3]);
+                for (int k = 0; k < 4; ++k) r[k] = __shfl_sync(0xffffffffu, own_row, (4 * lane + k) & 31);
+                if (lane < 8) {
+#pragma unroll
+                    for (int c = 0; c < kPanels; ++c)
+                        tma_gather4_pair(dst + c * kC2KPanel + lane * 512, &kv_map, bar, c * 64, r[0], r[1], r[2], r[3]);
                 }
             }
-            if (!ok) break;
             // advance the index pipeline: rows of tile i+1, page ids of tile i+2, positions of tile i+3
-            if (i + 1 < tiles) {
-                stage_rows(i + 1, own, a1, own_lo, own_hi, mask_own, contig, any_bad);
-                stage_rows(i + 1, oth, b1, oth_lo, oth_hi, mask_oth, contig_oth, any_bad);
-            }
-            a1 = a2;
-            b1 = b2;
-            stage_pages(a1);
-            stage_pages(b1);
-            stage_tokens(i + 3, own, a2);
-            stage_tokens(i + 3, oth, b2);
+            if (i + 1 < tiles) stage_rows(i + 1, x1, row_lo, row_hi, mask, contig, contig_lo, contig_hi, any_bad);
+            x1 = x2;
+            stage_pages(x1);
+            stage_tokens(i + 3, x2);
         }
         if (!ok && lane == 0) {
             flag_status(p.status, OMNI_DEV_TIMEOUT);
@@ -375,61 +340,91 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         if (__any_sync(0xffffffffu, any_bad) && lane == 0 && rank == 0) flag_status(p.status, OMNI_DEV_BAD_INDEX);
     } else if (warp == 6) {
         // =========================== V-role producer =====================================
+        // This CTA's V columns are [256*rank, 256*rank+256) = panels [4*rank, 4*rank+4) of all 64 tokens.
         bool any_bad = false;
-        HalfIdx x1[2], x2[2];
-        int lo[2], hi[2];
+        TileIdx x1, x2;
+        int row_lo, row_hi;
         uint64_t mask_unused;
-        bool contig[2];
-        for (int h = 0; h < 2; ++h) {
-            stage_tokens(0, h, x1[h]);
-            stage_pages(x1[h]);
-            stage_rows(0, h, x1[h], lo[h], hi[h], mask_unused, contig[h], any_bad);
-            stage_tokens(1, h, x1[h]);
-            stage_pages(x1[h]);
-            stage_tokens(2, h, x2[h]);
-        }
+        bool contig, contig_lo, contig_hi;
+        stage_tokens(0, x1);
+        stage_pages(x1);
+        stage_rows(0, x1, row_lo, row_hi, mask_unused, contig, contig_lo, contig_hi, any_bad);
+        stage_tokens(1, x1);
+        stage_pages(x1);
+        stage_tokens(2, x2);
         bool ok = true;
         for (int i = 0; ok && i < tiles; ++i) {
+            const int st = i & 1;
+            if (i >= 2) ok = mbar_wait(&ctl->pv_done[st], ((i >> 1) - 1) & 1);
+            ok = __all_sync(0xffffffffu, ok) && (*abort_flag == 0);
+            if (!ok) break;
+            const uint32_t bar = map_to_rank(smem_u32(&ctl->v_full[st]), 0);
+            if (lane == 0 && rank == 0) mbar_expect_tx(&ctl->v_full[st], 2 * kC2VBytes);
+            __syncwarp();
+            const uint32_t dst = smem_base + kC2SmemV + st * kC2VBytes;
+            if (contig) {
+                if (lane == 0) tma_box3d_pair(dst, &kv_v_map, bar, row_lo, 4 * (int)rank);
+            } else {
+                // lane g < 16 gathers tokens 4g..4g+3 into rows 4g..4g+3 of the four panels
+                int r[4];
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                if (i > 0) ok = mbar_wait(&ctl->v_empty[h], (i - 1) & 1);
-                ok = __all_sync(0xffffffffu, ok) && (*abort_flag == 0);
-                if (!ok) break;
-                const uint32_t bar = map_to_rank(smem_u32(&ctl->v_full[h]), 0);
-                if (lane == 0 && rank == 0) mbar_expect_tx(&ctl->v_full[h], 2 * kC2VHalfBytes);
-                __syncwarp();
-                const uint32_t dst = smem_base + kC2SmemV + h * kC2VHalfBytes;
-                if (contig[h]) {
-                    if (lane == 0) tma_box3d_pair(dst, &kv_v_map, bar, lo[h], 4 * (int)rank);
-                } else {
-                    int r[4];
-                    rows_of_four(lo[h], hi[h], r);
-                    if (lane < 16) {
+                for (int k = 0; k < 4; ++k) {
+                    const int src = (4 * lane + k) & 31;
+                    const int a = __shfl_sync(0xffffffffu, row_lo, src), c = __shfl_sync(0xffffffffu, row_hi, src);
+                    r[k] = lane < 8 ? a : c;
+                }
+                if (lane < 16) {
 #pragma unroll
-                        for (int c = 0; c < 4; ++c)
-                            tma_gather4_pair(dst + c * kPanelBytes + lane * 512, &kv_map, bar, ((int)rank * 4 + c) * 64, r[0],
-                                             r[1], r[2], r[3]);
-                    }
+                    for (int c = 0; c < 4; ++c)
+                        tma_gather4_pair(dst + c * kPanelBytes + lane * 512, &kv_map, bar, ((int)rank * 4 + c) * 64, r[0],
+                                         r[1], r[2], r[3]);
                 }
             }
-            if (!ok) break;
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                if (i + 1 < tiles) stage_rows(i + 1, h, x1[h], lo[h], hi[h], mask_unused, contig[h], any_bad);
-                x1[h] = x2[h];
-                stage_pages(x1[h]);
-                stage_tokens(i + 3, h, x2[h]);
-            }
+            if (i + 1 < tiles) stage_rows(i + 1, x1, row_lo, row_hi, mask_unused, contig, contig_lo, contig_hi, any_bad);
+            x1 = x2;
+            stage_pages(x1);
+            stage_tokens(i + 3, x2);
         }
         if (!ok && lane == 0) {
             flag_status(p.status, OMNI_DEV_TIMEOUT);
             *abort_flag = 1;
         }
+    } else if (warp == 7) {
+        // =========================== L2 prefetcher (CTA 0 only) ==========================
+        // A hint only: tiles that look like a whole page in order (first position page-aligned,
+        // last position 63 further) get their page prefetched into L2; anything else is left to
+        // the demand loads.  Lane l resolves tiles l, l+32, ... of a batch of 32 in parallel.
+        if (rank == 0) {
+            for (int t0 = 0; t0 < tiles; t0 += 32) {
+                const int t = t0 + lane;
+                const int j0 = begin + t * kC2Tile;
+                int row = -1;
+                if (t < tiles && j0 + kC2Tile <= end) {
+                    const int first = __ldg(sel + j0), last = __ldg(sel + j0 + kC2Tile - 1);
+                    if (first >= 0 && first % kPage == 0 && last == first + kC2Tile - 1 && first / kPage < p.max_pages) {
+                        const int pg = __ldg(pt + first / kPage);
+                        if (pg >= 0 && (int64_t)pg < p.num_pages) row = pg * kPage;
+                    }
+                }
+                const int count = min(32, tiles - t0);
+                bool ok = true;
+                for (int k = 0; ok && k < count; ++k) {
+                    const int i = t0 + k;
+                    if (i >= kPrefetchAhead + 2) {
+                        const int c = i - kPrefetchAhead;       // wait until Q K^T of tile c-2 retired
+                        ok = mbar_wait(&ctl->k_empty[c & 1], ((c >> 1) - 1) & 1);
+                        ok = __all_sync(0xffffffffu, ok) && (*abort_flag == 0);
+                    }
+                    if (ok && lane == k && row >= 0)
+                        asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(&kv_tile_map),
+                                     "r"(0), "r"(row), "r"(0)
+                                     : "memory");
+                }
+                if (!ok) break;
+            }
+        }
     } else if (warp == 1) {
         // =========================== MMA issuer (CTA 0 only) =============================
-        // The whole warp runs this loop with warp-uniform control flow and one elected lane issues
-        // each MMA / commit: descriptor arithmetic then stays cheap enough to issue an MMA every
-        // 32 clocks, which a lone diverged thread cannot.
         if (rank == 0) {
             constexpr uint32_t idesc_qk = instr_desc(128, kC2Tile, 0);
             constexpr uint32_t idesc_pv = instr_desc(128, 256, 1);
@@ -439,68 +434,76 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
             const uint64_t v_desc = smem_desc(smem_base + kC2SmemV, kPanelBytes, 1024);
             const uint32_t q_lo = (uint32_t)q_desc, k_lo = (uint32_t)k_desc, p_lo = (uint32_t)p_desc, v_lo = (uint32_t)v_desc;
             const uint32_t kmaj_hi = (uint32_t)(q_desc >> 32), v_hi = (uint32_t)(v_desc >> 32);
-            bool ok = mbar_wait(&ctl->q_full, 0);
-            int qk_t = 0, qk_c = 0, pv_t = 0, pv_h = 0;
-            long long idle_since = clock64();
-            while (ok && pv_t < tiles) {
-                bool progress = false;
-                // ---- one 64-token half of O += P V ----
-                if (pv_t < qk_t && (pv_h == 1 || mbar_test(&ctl->p_full, pv_t & 1)) &&
-                    mbar_test(&ctl->v_full[pv_h], pv_t & 1)) {
-                    tc_fence_after();
-                    const uint32_t a = p_lo + ((pv_h * kPanelBytes) >> 4);
-                    const uint32_t bd = v_lo + ((pv_h * kC2VHalfBytes) >> 4);
-                    if (pv_t == 0 && pv_h == 0) {
-                        tc_mma_pair_elect<false>(tmem + kColO, a, kmaj_hi, bd, v_hi, idesc_pv);
-                        tc_mma_pair_elect<false>(tmem + kColO + 128, a, kmaj_hi, bd + ((2 * kPanelBytes) >> 4), v_hi, idesc_pv);
-                    } else {
-                        tc_mma_pair_elect<true>(tmem + kColO, a, kmaj_hi, bd, v_hi, idesc_pv);
-                        tc_mma_pair_elect<true>(tmem + kColO + 128, a, kmaj_hi, bd + ((2 * kPanelBytes) >> 4), v_hi, idesc_pv);
-                    }
+            // Values that steer the loop are broadcast from lane 0 so that the compiler can see
+            // they are warp-uniform and keep the descriptor arithmetic on the uniform datapath;
+            // with thread-dependent control flow every MMA costs ~70 clocks to issue instead of ~25.
+            const int tiles_u = __shfl_sync(0xffffffffu, tiles, 0);
+            const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem, 0);
+            // The buffer parity is a compile-time constant of each issue routine (the tile loop is
+            // unrolled by two), so every operand of an MMA is a loop-invariant uniform value.
+            // S(t) = Q K(t)^T: 36 k-steps, Q panel c (8 KiB apart) against K panel c (4 KiB apart)
+            auto issue_qk = [&](auto par_tag) {
+                constexpr int par = decltype(par_tag)::value;
+                const uint32_t d = tmem_u + kC2ColS + 32 * par;
+                const uint32_t kb = k_lo + ((par * kC2KBytes) >> 4);
+                tc_mma_pair_elect<false>(d, q_lo, kmaj_hi, kb, kmaj_hi, idesc_qk);
 #pragma unroll
-                    for (int k = 1; k < 4; ++k) {
-                        const uint32_t ak = a + ((k * 32) >> 4), bk = bd + ((k * 2048) >> 4);
-                        tc_mma_pair_elect<true>(tmem + kColO, ak, kmaj_hi, bk, v_hi, idesc_pv);
-                        tc_mma_pair_elect<true>(tmem + kColO + 128, ak, kmaj_hi, bk + ((2 * kPanelBytes) >> 4), v_hi, idesc_pv);
-                    }
-                    tc_commit_pair_elect(&ctl->v_empty[pv_h]);
-                    if (pv_h == 1) {
-                        tc_commit_pair_elect(&ctl->pv_done);
-                        ++pv_t;
-                        pv_h = 0;
-                    } else {
-                        pv_h = 1;
-                    }
-                    progress = true;
+                for (int kk = 1; kk < kDqk / 16; ++kk)
+                    tc_mma_pair_elect<true>(d, q_lo + (((kk >> 2) * kPanelBytes + (kk & 3) * 32) >> 4), kmaj_hi,
+                                            kb + (((kk >> 2) * kC2KPanel + (kk & 3) * 32) >> 4), kmaj_hi, idesc_qk);
+                tc_commit_pair_elect(&ctl->k_empty[par]);
+                tc_commit_pair_elect(&ctl->s_full[par]);
+            };
+            // O += P(t) V(t): 4 k-steps of 16 tokens, two N=256 instructions each
+            auto issue_pv = [&](auto par_tag, bool first) {
+                constexpr int par = decltype(par_tag)::value;
+                const uint32_t a = p_lo + ((par * kPanelBytes) >> 4);
+                const uint32_t bd = v_lo + ((par * kC2VBytes) >> 4);
+                if (first) {
+                    tc_mma_pair_elect<false>(tmem_u + kColO, a, kmaj_hi, bd, v_hi, idesc_pv);
+                    tc_mma_pair_elect<false>(tmem_u + kColO + 128, a, kmaj_hi, bd + ((2 * kPanelBytes) >> 4), v_hi, idesc_pv);
+                } else {
+                    tc_mma_pair_elect<true>(tmem_u + kColO, a, kmaj_hi, bd, v_hi, idesc_pv);
+                    tc_mma_pair_elect<true>(tmem_u + kColO + 128, a, kmaj_hi, bd + ((2 * kPanelBytes) >> 4), v_hi, idesc_pv);
                 }
-                // ---- one group of three 64-column panels of S = Q K^T ----
-                if (qk_t < tiles && mbar_test(&ctl->k_full[qk_c], qk_t & 1) &&
-                    (qk_c > 0 || qk_t < 2 || mbar_test(&ctl->s_empty[qk_t & 1], ((qk_t >> 1) - 1) & 1))) {
-                    tc_fence_after();
-                    const uint32_t d = tmem + kC2ColS + 64 * (qk_t & 1);
-                    const uint32_t off = (qk_c * kKGroupBytes) >> 4;
-                    if (qk_c == 0)
-                        tc_mma_pair_elect<false>(d, q_lo, kmaj_hi, k_lo, kmaj_hi, idesc_qk);
-                    else
-                        tc_mma_pair_elect<true>(d, q_lo + off, kmaj_hi, k_lo + off, kmaj_hi, idesc_qk);
 #pragma unroll
-                    for (int k = 1; k < 12; ++k) {
-                        const uint32_t o = off + (((k >> 2) * kPanelBytes + (k & 3) * 32) >> 4);
-                        tc_mma_pair_elect<true>(d, q_lo + o, kmaj_hi, k_lo + o, kmaj_hi, idesc_qk);
-                    }
-                    tc_commit_pair_elect(&ctl->k_empty[qk_c]);
-                    if (++qk_c == kKGroups) {
-                        tc_commit_pair_elect(&ctl->s_full[qk_t & 1]);
-                        qk_c = 0;
-                        ++qk_t;
-                    }
-                    progress = true;
+                for (int k = 1; k < 4; ++k) {
+                    const uint32_t ak = a + ((k * 32) >> 4), bk = bd + ((k * 2048) >> 4);
+                    tc_mma_pair_elect<true>(tmem_u + kColO, ak, kmaj_hi, bk, v_hi, idesc_pv);
+                    tc_mma_pair_elect<true>(tmem_u + kColO + 128, ak, kmaj_hi, bk + ((2 * kPanelBytes) >> 4), v_hi, idesc_pv);
                 }
-                if (progress)
-                    idle_since = clock64();
-                else if (clock64() - idle_since > kWaitCycles || *abort_flag)
-                    ok = false;
-                ok = __all_sync(0xffffffffu, ok);
+                tc_commit_pair_elect(&ctl->pv_done[par]);
+            };
+            // one tile: Q K^T of the NEXT tile first (its K was requested two tiles ago, so the wait
+            // is normally already satisfied), then P V of this tile
+            auto step = [&](auto par_tag, int i) -> bool {
+                constexpr int par = decltype(par_tag)::value;
+                bool good = true;
+                if (i + 1 < tiles_u) {
+                    const int t = i + 1;
+                    good = mbar_wait(&ctl->k_full[par ^ 1], (t >> 1) & 1) &&
+                           (t < 2 || mbar_wait(&ctl->s_empty[par ^ 1], ((t >> 1) - 1) & 1));
+                    good = __all_sync(0xffffffffu, good);
+                    if (!good) return false;
+                    tc_fence_after();
+                    issue_qk(std::integral_constant<int, par ^ 1>{});
+                }
+                good = mbar_wait(&ctl->p_full[par], (i >> 1) & 1) && mbar_wait(&ctl->v_full[par], (i >> 1) & 1);
+                good = __all_sync(0xffffffffu, good);
+                if (!good) return false;
+                tc_fence_after();
+                issue_pv(par_tag, i == 0);
+                return true;
+            };
+            bool ok = mbar_wait(&ctl->q_full, 0) && mbar_wait(&ctl->k_full[0], 0);
+            ok = __all_sync(0xffffffffu, ok);
+            if (ok) {
+                tc_fence_after();
+                issue_qk(std::integral_constant<int, 0>{});
+            }
+            for (int i = 0; ok && i < tiles_u; i += 2) {
+                ok = step(std::integral_constant<int, 0>{}, i);
+                if (ok && i + 1 < tiles_u) ok = step(std::integral_constant<int, 1>{}, i + 1);
             }
             if (!ok && lane == 0) {
                 flag_status(p.status, OMNI_DEV_TIMEOUT);
@@ -514,10 +517,10 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         const int row = (quarter & 1) * 32 + lane;          // head row within this CTA
         const int half = quarter >> 1;                      // token half of S / column half of O
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-        const uint32_t s_empty0 = map_to_rank(smem_u32(&ctl->s_empty[0]), 0);
-        const uint32_t s_empty1 = map_to_rank(smem_u32(&ctl->s_empty[1]), 0);
-        const uint32_t p_full_leader = map_to_rank(smem_u32(&ctl->p_full), 0);
-        uint8_t *p_row = smem + kC2SmemP + half * kPanelBytes + row * 128;
+        const uint32_t s_empty_leader[2] = {map_to_rank(smem_u32(&ctl->s_empty[0]), 0),
+                                            map_to_rank(smem_u32(&ctl->s_empty[1]), 0)};
+        const uint32_t p_full_leader[2] = {map_to_rank(smem_u32(&ctl->p_full[0]), 0),
+                                           map_to_rank(smem_u32(&ctl->p_full[1]), 0)};
         float m_ref = -INFINITY, l = 0.f;
         bool ok = true;
         for (int i = 0; i < tiles; ++i) {
@@ -528,20 +531,27 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
                 break;
             }
             tc_fence_after();
-            uint32_t sv[64];
-            tc_ld32(tmem + lane_base + kC2ColS + 64 * buf, *reinterpret_cast<uint32_t(*)[32]>(&sv[0]));
-            tc_ld32(tmem + lane_base + kC2ColS + 64 * buf + 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[32]));
+            uint32_t sv[32];
+            tc_ld32(tmem + lane_base + kC2ColS + 32 * buf, sv);
             tc_wait_ld();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(buf ? s_empty1 : s_empty0);
-            const uint64_t valid = ctl->valid_mask[i % kMaskRing][half];
+            if (lane == 0) mbar_arrive_cluster(s_empty_leader[buf]);
+            const uint32_t valid = (uint32_t)(ctl->valid_mask[i % kMaskRing] >> (32 * half));
+            float x[32];
             float mt = -INFINITY;
+            if (valid == 0xffffffffu) {
 #pragma unroll
-            for (int j = 0; j < 64; ++j) {
-                const float x = ((valid >> j) & 1ull) ? __uint_as_float(sv[j]) * p.scale_log2 : -INFINITY;
-                sv[j] = __float_as_uint(x);
-                mt = fmaxf(mt, x);
+                for (int j = 0; j < 32; ++j) {
+                    x[j] = __uint_as_float(sv[j]) * p.scale_log2;
+                    mt = fmaxf(mt, x[j]);
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    x[j] = ((valid >> j) & 1u) ? __uint_as_float(sv[j]) * p.scale_log2 : -INFINITY;
+                    mt = fmaxf(mt, x[j]);
+                }
             }
             // the other token half of this row lives in the warp two quarters away
             ctl->xchg[i & 1][half][row] = mt;
@@ -561,48 +571,55 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
             }
             const float mr = (m_ref == -INFINITY) ? 0.f : m_ref;
             float sum = 0.f;
-            uint32_t pk[32];
+            uint32_t pk[16];
 #pragma unroll
-            for (int j = 0; j < 64; j += 2) {
-                const float e0 = exp2f(__uint_as_float(sv[j]) - mr), e1 = exp2f(__uint_as_float(sv[j + 1]) - mr);
+            for (int j = 0; j < 32; j += 2) {
+                const float e0 = exp2f(x[j] - mr), e1 = exp2f(x[j + 1] - mr);
                 sum += e0 + e1;
                 pk[j >> 1] = pack_bf16(e0, e1);
             }
             l = l * factor + sum;
-            if (i > 0) {
-                ok = mbar_wait(&ctl->pv_done, (i - 1) & 1);
+            // the P buffer is free once P V of tile i-2 retired; O may be rescaled once P V of tile i-1 did
+            if (i >= 2) {
+                ok = mbar_wait(&ctl->pv_done[buf], ((i >> 1) - 1) & 1);
+                if (!__all_sync(0xffffffffu, ok)) {
+                    ok = false;
+                    break;
+                }
+            }
+            if (i >= 1 && __any_sync(0xffffffffu, moved)) {
+                ok = mbar_wait(&ctl->pv_done[buf ^ 1], ((i - 1) >> 1) & 1);
                 if (!__all_sync(0xffffffffu, ok)) {
                     ok = false;
                     break;
                 }
                 tc_fence_after();
-                if (__any_sync(0xffffffffu, moved)) {
 #pragma unroll 1
-                    for (int c = 0; c < 256; c += 32) {
-                        uint32_t ov[32];
-                        tc_ld32(tmem + lane_base + kColO + c, ov);
-                        tc_wait_ld();
+                for (int c = 0; c < 256; c += 32) {
+                    uint32_t ov[32];
+                    tc_ld32(tmem + lane_base + kColO + c, ov);
+                    tc_wait_ld();
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * factor);
-                        tc_st32(tmem + lane_base + kColO + c, ov);
-                    }
-                    tc_wait_st();
+                    for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * factor);
+                    tc_st32(tmem + lane_base + kColO + c, ov);
                 }
+                tc_wait_st();
             }
-            // P row half: 64 tokens x bf16 = 128 B = eight 16-byte chunks, chunk c stored at c ^ (row % 8)
+            // P row half: 32 tokens x bf16 = 64 B = four 16-byte chunks, chunk c stored at c ^ (row % 8)
+            uint8_t *p_row = smem + kC2SmemP + buf * kPanelBytes + row * 128;
 #pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                const int chunk = c ^ (row & 7);
+            for (int c = 0; c < 4; ++c) {
+                const int chunk = (half * 4 + c) ^ (row & 7);
                 *reinterpret_cast<uint4 *>(p_row + chunk * 16) =
                     make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
             }
             fence_async_smem();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(p_full_leader);
+            if (lane == 0) mbar_arrive_cluster(p_full_leader[buf]);
         }
         if (ok) {
-            ok = mbar_wait(&ctl->pv_done, (tiles - 1) & 1);
+            ok = mbar_wait(&ctl->pv_done[(tiles - 1) & 1], ((tiles - 1) >> 1) & 1);
             ok = __all_sync(0xffffffffu, ok);
         }
         if (ok) {
@@ -613,23 +630,27 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
             ok = __all_sync(0xffffffffu, ok);
         }
         if (ok) {
+            // The 64 output rows of this CTA are one contiguous block of global memory.  They are
+            // staged in shared memory (all operand buffers are dead by now; the row pitch is padded
+            // by 16 B so that the 32 rows a warp writes at once fall in different banks) and leave
+            // as one bulk copy per row: full-line writes instead of scattered 16-byte stores.
             tc_fence_after();
             const float lt = l + ctl->xchg[tiles & 1][half ^ 1][row];
             const float inv = lt > 0.f ? 1.f / lt : 0.f;
             const int h = h0 + row;
             const bool store = h < p.heads;
-            const size_t u = p.splits == 1 ? ((size_t)b * p.heads + h) : (((size_t)b * p.splits + s) * p.heads + h);
+            const bool final_out = p.splits == 1;
+            const size_t u = final_out ? ((size_t)b * p.heads + h) : (((size_t)b * p.splits + s) * p.heads + h);
+            const uint32_t row_bytes = final_out ? kDv * 2 : kDv * 4, pitch = row_bytes + 16;
+            uint8_t *stage_row = smem + (size_t)row * pitch + half * (row_bytes / 2);
 #pragma unroll 1
             for (int c = 0; c < 256; c += 32) {
                 uint32_t ov[32];
                 __syncwarp();
                 tc_ld32(tmem + lane_base + kColO + c, ov);
                 tc_wait_ld();
-                const int col = half * 256 + c;
-                if (!store) {
-                    // padded head row: nothing to write
-                } else if (p.splits == 1) {
-                    uint4 *o = reinterpret_cast<uint4 *>(p.out + u * kDv + col);
+                if (final_out) {
+                    uint4 *o = reinterpret_cast<uint4 *>(stage_row + c * 2);
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         uint4 w;
@@ -640,7 +661,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
                         o[j] = w;
                     }
                 } else {
-                    float4 *o = reinterpret_cast<float4 *>(p.part_out + u * kDv + col);
+                    float4 *o = reinterpret_cast<float4 *>(stage_row + c * 4);
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
                         o[j] = make_float4(__uint_as_float(ov[4 * j]) * inv, __uint_as_float(ov[4 * j + 1]) * inv,
@@ -649,12 +670,27 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
             }
             if (store && half == 0) {
                 const float lse = lt > 0.f ? (m_ref + log2f(lt)) * kLn2 : -INFINITY;
-                if (p.splits == 1)
+                if (final_out)
                     p.lse[u] = lse;
                 else
                     p.part_lse[u] = lse;
             }
-        } else if (lane == 0) {
+            // both halves of every row staged -> the thread that owns the first half sends the row
+            fence_async_smem();
+            mbar_arrive(&ctl->x_bar);
+            ok = mbar_wait(&ctl->x_bar, (tiles + 1) & 1);
+            ok = __all_sync(0xffffffffu, ok);
+            if (ok && store && half == 0) {
+                uint8_t *dst = final_out ? reinterpret_cast<uint8_t *>(p.out + u * kDv)
+                                         : reinterpret_cast<uint8_t *>(p.part_out + u * kDv);
+                asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst),
+                             "r"(smem_u32(smem + (size_t)row * pitch)), "r"(row_bytes)
+                             : "memory");
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+            }
+        }
+        if (!ok && lane == 0) {
             flag_status(p.status, OMNI_DEV_TIMEOUT);
             *abort_flag = 1;
         }
@@ -667,8 +703,17 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     }
     tc_fence_before();
     __syncthreads();
-    cluster_sync_all();
+    // Tensor memory was allocated for the pair, so it is released only when both CTAs are done
+    // with it.  The rendezvous is an mbarrier in each CTA that both CTAs arrive on (the hardware
+    // cluster barrier took 6-9 us at this point); warp 1 stays until the peer's arrival has
+    // landed, which also keeps this CTA's shared memory alive for it.
+    if (threadIdx.x == 0) {
+        mbar_arrive(&ctl->exit_bar);
+        mbar_arrive_cluster(map_to_rank(smem_u32(&ctl->exit_bar), rank ^ 1));
+    }
     if (warp == 1) {
+        mbar_wait(&ctl->exit_bar, 0);
+        __syncwarp();
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
@@ -685,11 +730,12 @@ inline omni_status_t launch_tc2_decode(const DecodeParams &p, cudaStream_t strea
             return OMNI_ERR_CUDA;
         attr_set[dev] = true;
     }
-    CUtensorMap q_map, kv_map, kv_k_map, kv_v_map;
-    if (!make_panel_map(&q_map, p.q, (uint64_t)p.batch * p.heads, kPanels)) return OMNI_ERR_CUDA;
+    CUtensorMap q_map, kv_map, kv_k_map, kv_v_map, kv_tile_map;
+    if (!make_panel_map(&kv_tile_map, p.kv, (uint64_t)p.num_pages * kPage, kTile, kPanels)) return OMNI_ERR_CUDA;
+    if (!make_panel_map(&q_map, p.q, (uint64_t)p.batch * p.heads, kTcHeads, kPanels)) return OMNI_ERR_CUDA;
     if (!make_row_map(&kv_map, p.kv, (uint64_t)p.num_pages * kPage, 1)) return OMNI_ERR_CUDA;
-    if (!make_panel_map(&kv_k_map, p.kv, (uint64_t)p.num_pages * kPage, 3)) return OMNI_ERR_CUDA;
-    if (!make_panel_map(&kv_v_map, p.kv, (uint64_t)p.num_pages * kPage, 4)) return OMNI_ERR_CUDA;
+    if (!make_panel_map(&kv_k_map, p.kv, (uint64_t)p.num_pages * kPage, 32, kPanels)) return OMNI_ERR_CUDA;
+    if (!make_panel_map(&kv_v_map, p.kv, (uint64_t)p.num_pages * kPage, kTile, 4)) return OMNI_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(p.batch * p.splits * 2));
     cfg.blockDim = dim3(kC2Threads);
@@ -702,8 +748,9 @@ inline omni_status_t launch_tc2_decode(const DecodeParams &p, cudaStream_t strea
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, tc2_decode_kernel, q_map, kv_map, kv_k_map, kv_v_map, p) == cudaSuccess ? OMNI_OK
-                                                                                                      : OMNI_ERR_CUDA;
+    return cudaLaunchKernelEx(&cfg, tc2_decode_kernel, q_map, kv_map, kv_k_map, kv_v_map, kv_tile_map, p) == cudaSuccess
+               ? OMNI_OK
+               : OMNI_ERR_CUDA;
 }
 
 }  // namespace omni

@@ -24,6 +24,8 @@
 
 #include <cuda.h>
 
+#include <mutex>
+
 #include "common.cuh"
 
 namespace omni {
@@ -644,8 +646,46 @@ inline EncodeTiledFn encode_tiled_fn()
     return fn;
 }
 
+// Encoding a tensor map costs about a microsecond of host time and a decode step needs up to
+// five, more than the launch itself, so the most recent encodings are kept (a map depends only
+// on the base address and the sizes; nothing in it refers to a call).
+struct MapCacheEntry {
+    const void *base;
+    uint64_t rows;
+    uint32_t box_rows, box_panels, kind;
+    CUtensorMap map;
+};
+
+inline bool cached_map(CUtensorMap *out, const void *base, uint64_t rows, uint32_t box_rows, uint32_t box_panels,
+                       uint32_t kind, bool (*encode)(CUtensorMap *, const void *, uint64_t, uint32_t, uint32_t))
+{
+    constexpr int kEntries = 32;
+    static MapCacheEntry cache[kEntries];
+    static int used = 0, next = 0;
+    static std::mutex mu;
+    std::lock_guard<std::mutex> lock(mu);
+    for (int i = 0; i < used; ++i) {
+        const MapCacheEntry &e = cache[i];
+        if (e.base == base && e.rows == rows && e.box_rows == box_rows && e.box_panels == box_panels && e.kind == kind) {
+            *out = e.map;
+            return true;
+        }
+    }
+    if (!encode(out, base, rows, box_rows, box_panels)) return false;
+    MapCacheEntry &e = cache[next];
+    e.base = base;
+    e.rows = rows;
+    e.box_rows = box_rows;
+    e.box_panels = box_panels;
+    e.kind = kind;
+    e.map = *out;
+    next = (next + 1) % kEntries;
+    if (used < kEntries) ++used;
+    return true;
+}
+
 // 2-D bf16 row-major [rows, 576] tensor, boxes of 64 columns x box_rows rows, 128-byte swizzle.
-inline bool make_row_map(CUtensorMap *map, const void *base, uint64_t rows, uint32_t box_rows)
+inline bool encode_row_map(CUtensorMap *map, const void *base, uint64_t rows, uint32_t box_rows, uint32_t)
 {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
@@ -658,20 +698,30 @@ inline bool make_row_map(CUtensorMap *map, const void *base, uint64_t rows, uint
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// The same tensor seen as [rows, 9 panels of 64 columns]: 3-D boxes {64 columns, 64 rows, n panels}
+// The same tensor seen as [rows, 9 panels of 64 columns]: 3-D boxes {64 columns, box_rows, n panels}
 // land in shared memory panel by panel ([64 rows x 128 B] each, 128-byte swizzle), which is the
 // operand layout of the MMAs, so one instruction fills up to a whole 72 KiB tile.
-inline bool make_panel_map(CUtensorMap *map, const void *base, uint64_t rows, uint32_t box_panels)
+inline bool encode_panel_map(CUtensorMap *map, const void *base, uint64_t rows, uint32_t box_rows, uint32_t box_panels)
 {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
     const cuuint64_t dims[3] = {64, (cuuint64_t)rows, (cuuint64_t)kPanels};
     const cuuint64_t strides[2] = {(cuuint64_t)kDqk * 2, 128};
-    const cuuint32_t box[3] = {64, (cuuint32_t)kTile, box_panels};
+    const cuuint32_t box[3] = {64, box_rows, box_panels};
     const cuuint32_t estr[3] = {1, 1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+inline bool make_row_map(CUtensorMap *map, const void *base, uint64_t rows, uint32_t box_rows)
+{
+    return cached_map(map, base, rows, box_rows, 0, 0, encode_row_map);
+}
+
+inline bool make_panel_map(CUtensorMap *map, const void *base, uint64_t rows, uint32_t box_rows, uint32_t box_panels)
+{
+    return cached_map(map, base, rows, box_rows, box_panels, 1, encode_panel_map);
 }
 
 inline omni_status_t launch_tc_decode(const DecodeParams &p, cudaStream_t stream)
