@@ -25,6 +25,7 @@
 #include <cuda.h>
 
 #include <mutex>
+#include <type_traits>
 
 #include "common.cuh"
 
@@ -122,6 +123,16 @@ __device__ __forceinline__ void tma_box2d(uint32_t dst, const CUtensorMap *map, 
         "cp.async.bulk.tensor.2d.shared::cta.global.tile.mbarrier::complete_tx::bytes"
         " [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(map), "r"(col), "r"(row), "r"(smem_u32(bar))
+        : "memory");
+}
+
+// 3-D box {64 columns, rows, panels} of the [rows, 9 panels, 64 columns] view: lands panel by panel.
+__device__ __forceinline__ void tma_box3d(uint32_t dst, const CUtensorMap *map, uint64_t *bar, int row, int panel)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cta.global.tile.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(map), "r"(0), "r"(row), "r"(panel), "r"(smem_u32(bar))
         : "memory");
 }
 
@@ -229,6 +240,33 @@ __device__ __forceinline__ void tc_mma_c(uint32_t d_tmem, uint64_t a_desc, uint6
         : "memory");
 }
 
+// MMA / commit executed by a whole converged warp: one elected lane issues the instruction.  The
+// descriptors arrive as 32-bit halves so that stepping through a tile is a 32-bit add.
+template <bool kAccumulate>
+__device__ __forceinline__ void tc_mma_elect(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                             uint32_t idesc)
+{
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t.reg .b64 da, db;\n\t"
+        "mov.b64 da, {%1, %2};\n\t"
+        "mov.b64 db, {%3, %4};\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "elect.sync _|q, 0xffffffff;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "n"(kAccumulate ? 1 : 0)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_commit_elect(uint64_t *bar)
+{
+    asm volatile(
+        "{\n\t.reg .pred q;\n\t"
+        "elect.sync _|q, 0xffffffff;\n\t"
+        "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+        ::"r"(smem_u32(bar))
+        : "memory");
+}
+
 // 16 lanes x 32 columns twice: threads 0-15 of the warp read columns [c, c+32) of lanes 0-15 of
 // their quarter, threads 16-31 read columns [c+32, c+64) of the same lanes.  This is how the 64
 // rows of an M=64 accumulator (which live in lanes 0-15 of each quarter) are spread over all 32
@@ -260,7 +298,7 @@ tc_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constan
     const int hg = blockIdx.x % head_groups;
     const int s = (blockIdx.x / head_groups) % p.splits;
     const int b = blockIdx.x / (head_groups * p.splits);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;  // warp-uniform
     const int h0 = hg * kTcHeads;
 
     int n = __ldg(p.sel_len + b);
@@ -327,8 +365,7 @@ tc_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constan
         const int32_t *pt = p.page_table + (size_t)b * p.max_pages;
         if (lane == 0) {
             mbar_expect_tx(&ctl->q_full, kTileBytes);
-            for (int c = 0; c < kPanels; ++c)
-                tma_box2d(smem_base + kSmemQ + c * kPanelBytes, &q_map, &ctl->q_full, c * 64, b * p.heads + h0);
+            tma_box3d(smem_base + kSmemQ, &q_map, &ctl->q_full, b * p.heads + h0, 0);
         }
         bool any_bad = bad_len;
         // Lane l serves tokens l and l+32 of a tile.  Token positions are fetched two tiles
@@ -383,9 +420,8 @@ tc_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constan
             __syncwarp();
             const uint32_t stage = smem_base + kSmemKV + st * kTileBytes;
             if (contig) {
-                // 64 consecutive pool rows (a whole page in order): one 64x64 box per column panel
-                if (lane < kPanels)
-                    tma_box2d(stage + lane * kPanelBytes, &kv_page_map, &ctl->kv_full[st], lane * 64, row_lo - lane);
+                // 64 consecutive pool rows (a whole page in order): the whole tile is one 3-D box
+                if (lane == 0) tma_box3d(stage, &kv_page_map, &ctl->kv_full[st], row_lo, 0);
             } else {
                 // scattered rows: lane g < 16 gathers tokens 4g..4g+3 into rows 4g..4g+3 of every panel
                 int r[4];
@@ -414,70 +450,86 @@ tc_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constan
         }
     } else if (warp == 1) {
         // =========================== MMA issuer =========================================
-        if (lane == 0) {
+        // The whole warp runs this loop with warp-uniform control flow (loop bounds broadcast from
+        // lane 0, buffer parity a compile-time constant) and one elected lane issues each MMA: the
+        // descriptor arithmetic then stays on the uniform datapath and an MMA issues every ~30 clocks,
+        // where a lone diverged thread needs ~75.
+        {
             constexpr uint32_t idesc_qk = instr_desc(kTcHeads, kTile, 0);
             constexpr uint32_t idesc_pv = instr_desc(kTcHeads, 256, 1);
             const uint64_t q_desc = smem_desc(smem_base + kSmemQ, 16, 1024);
+            const uint64_t k_desc = smem_desc(smem_base + kSmemKV, 16, 1024);
             const uint64_t p_desc = smem_desc(smem_base + kSmemP, 16, 1024);
-            bool ok = mbar_wait(&ctl->q_full, 0);
+            const uint64_t v_desc = smem_desc(smem_base + kSmemKV, kPanelBytes, 1024);
+            const uint32_t q_lo = (uint32_t)q_desc, k_lo = (uint32_t)k_desc, p_lo = (uint32_t)p_desc, v_lo = (uint32_t)v_desc;
+            const uint32_t kmaj_hi = (uint32_t)(q_desc >> 32), v_hi = (uint32_t)(v_desc >> 32);
+            const int tiles_u = __shfl_sync(0xffffffffu, tiles, 0);
+            const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem, 0);
             // S(t) = Q K(t)^T : 36 k-steps of 16 columns; panel c of Q against panel c of the stage
-            auto issue_qk = [&](int t) {
-                const uint64_t k_desc = smem_desc(smem_base + kSmemKV + (t % kStages) * kTileBytes, 16, 1024);
-                const uint32_t d = tmem + kColS + 64 * (t & 1);
-                tc_mma_c<false>(d, q_desc, k_desc, idesc_qk);
+            auto issue_qk = [&](auto par_tag) {
+                constexpr int par = decltype(par_tag)::value;
+                const uint32_t d = tmem_u + kColS + 64 * par;
+                const uint32_t kb = k_lo + ((par * kTileBytes) >> 4);
+                tc_mma_elect<false>(d, q_lo, kmaj_hi, kb, kmaj_hi, idesc_qk);
 #pragma unroll
                 for (int kk = 1; kk < kDqk / 16; ++kk) {
                     const uint32_t off = ((kk >> 2) * kPanelBytes + (kk & 3) * 32) >> 4;
-                    tc_mma_c<true>(d, q_desc + off, k_desc + off, idesc_qk);
+                    tc_mma_elect<true>(d, q_lo + off, kmaj_hi, kb + off, kmaj_hi, idesc_qk);
                 }
-                tc_commit(&ctl->s_full[t & 1]);
+                tc_commit_elect(&ctl->s_full[par]);
             };
             // O += P(i) V(i) : the stage read N-major (64-column panels 8192 B apart, 8-token groups
             // 1024 B apart); value columns 0..255 and 256..511 go to the two interleaved accumulators
-            auto issue_pv = [&](int i) {
-                const uint64_t v_desc = smem_desc(smem_base + kSmemKV + (i % kStages) * kTileBytes, kPanelBytes, 1024);
-                if (i == 0) {
-                    tc_mma_c<false>(tmem + kColO, p_desc, v_desc, idesc_pv);
-                    tc_mma_c<false>(tmem + kColO + kLane16, p_desc, v_desc + ((4 * kPanelBytes) >> 4), idesc_pv);
+            auto issue_pv = [&](auto par_tag, bool first) {
+                constexpr int par = decltype(par_tag)::value;
+                const uint32_t vb = v_lo + ((par * kTileBytes) >> 4);
+                if (first) {
+                    tc_mma_elect<false>(tmem_u + kColO, p_lo, kmaj_hi, vb, v_hi, idesc_pv);
+                    tc_mma_elect<false>(tmem_u + kColO + kLane16, p_lo, kmaj_hi, vb + ((4 * kPanelBytes) >> 4), v_hi, idesc_pv);
                 } else {
-                    tc_mma_c<true>(tmem + kColO, p_desc, v_desc, idesc_pv);
-                    tc_mma_c<true>(tmem + kColO + kLane16, p_desc, v_desc + ((4 * kPanelBytes) >> 4), idesc_pv);
+                    tc_mma_elect<true>(tmem_u + kColO, p_lo, kmaj_hi, vb, v_hi, idesc_pv);
+                    tc_mma_elect<true>(tmem_u + kColO + kLane16, p_lo, kmaj_hi, vb + ((4 * kPanelBytes) >> 4), v_hi, idesc_pv);
                 }
 #pragma unroll
                 for (int k = 1; k < kTile / 16; ++k) {
-                    tc_mma_c<true>(tmem + kColO, p_desc + ((k * 32) >> 4), v_desc + ((k * 2048) >> 4), idesc_pv);
-                    tc_mma_c<true>(tmem + kColO + kLane16, p_desc + ((k * 32) >> 4),
-                                   v_desc + ((4 * kPanelBytes + k * 2048) >> 4), idesc_pv);
+                    tc_mma_elect<true>(tmem_u + kColO, p_lo + ((k * 32) >> 4), kmaj_hi, vb + ((k * 2048) >> 4), v_hi, idesc_pv);
+                    tc_mma_elect<true>(tmem_u + kColO + kLane16, p_lo + ((k * 32) >> 4), kmaj_hi,
+                                       vb + ((4 * kPanelBytes + k * 2048) >> 4), v_hi, idesc_pv);
                 }
-                tc_commit(&ctl->kv_empty[i % kStages]);
-                tc_commit(&ctl->pv_done);
+                tc_commit_elect(&ctl->kv_empty[par]);
+                tc_commit_elect(&ctl->pv_done);
             };
-            // Issue whichever of "next Q K^T" and "next P V" has its inputs ready, so a late tile
-            // never holds back the P V that frees a stage.
-            int next_qk = 0, next_pv = 0;
-            long long idle_since = clock64();
-            while (ok && next_pv < tiles) {
-                bool progress = false;
-                if (next_qk < tiles && next_qk <= next_pv + 1 &&
-                    mbar_test(&ctl->kv_full[next_qk % kStages], (next_qk / kStages) & 1) &&
-                    (next_qk < 2 || mbar_test(&ctl->s_empty[next_qk & 1], ((next_qk >> 1) - 1) & 1))) {
+            // one tile: Q K^T of the next tile first, then P V of this one
+            auto step = [&](auto par_tag, int i) -> bool {
+                constexpr int par = decltype(par_tag)::value;
+                bool good = true;
+                if (i + 1 < tiles_u) {
+                    const int t = i + 1;
+                    good = mbar_wait(&ctl->kv_full[par ^ 1], (t >> 1) & 1) &&
+                           (t < 2 || mbar_wait(&ctl->s_empty[par ^ 1], ((t >> 1) - 1) & 1));
+                    good = __all_sync(0xffffffffu, good);
+                    if (!good) return false;
                     tc_fence_after();
-                    issue_qk(next_qk);
-                    ++next_qk;
-                    progress = true;
+                    issue_qk(std::integral_constant<int, par ^ 1>{});
                 }
-                if (next_pv < next_qk && mbar_test(&ctl->p_full, next_pv & 1)) {
-                    tc_fence_after();
-                    issue_pv(next_pv);
-                    ++next_pv;
-                    progress = true;
-                }
-                if (progress)
-                    idle_since = clock64();
-                else if (clock64() - idle_since > kWaitCycles || *abort_flag)
-                    ok = false;
+                good = mbar_wait(&ctl->p_full, i & 1);
+                good = __all_sync(0xffffffffu, good);
+                if (!good) return false;
+                tc_fence_after();
+                issue_pv(par_tag, i == 0);
+                return true;
+            };
+            bool ok = mbar_wait(&ctl->q_full, 0) && mbar_wait(&ctl->kv_full[0], 0);
+            ok = __all_sync(0xffffffffu, ok);
+            if (ok) {
+                tc_fence_after();
+                issue_qk(std::integral_constant<int, 0>{});
             }
-            if (!ok) {
+            for (int i = 0; ok && i < tiles_u; i += 2) {
+                ok = step(std::integral_constant<int, 0>{}, i);
+                if (ok && i + 1 < tiles_u) ok = step(std::integral_constant<int, 1>{}, i + 1);
+            }
+            if (!ok && lane == 0) {
                 flag_status(p.status, OMNI_DEV_TIMEOUT);
                 *abort_flag = 1;
             }
@@ -736,9 +788,9 @@ inline omni_status_t launch_tc_decode(const DecodeParams &p, cudaStream_t stream
         attr_set[dev] = true;
     }
     CUtensorMap q_map, kv_map, kv_page_map;
-    if (!make_row_map(&q_map, p.q, (uint64_t)p.batch * p.heads, kTcHeads)) return OMNI_ERR_CUDA;
+    if (!make_panel_map(&q_map, p.q, (uint64_t)p.batch * p.heads, kTcHeads, kPanels)) return OMNI_ERR_CUDA;
     if (!make_row_map(&kv_map, p.kv, (uint64_t)p.num_pages * kPage, 1)) return OMNI_ERR_CUDA;
-    if (!make_row_map(&kv_page_map, p.kv, (uint64_t)p.num_pages * kPage, kTile)) return OMNI_ERR_CUDA;
+    if (!make_panel_map(&kv_page_map, p.kv, (uint64_t)p.num_pages * kPage, kTile, kPanels)) return OMNI_ERR_CUDA;
     const int head_groups = (p.heads + kTcHeads - 1) / kTcHeads;
     const unsigned grid = (unsigned)(p.batch * p.splits * head_groups);
     tc_decode_kernel<<<grid, kTcThreads, kTcSmemBytes, stream>>>(q_map, kv_map, kv_page_map, p);
