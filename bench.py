@@ -148,6 +148,36 @@ def _oracle_sample(w, target_s=15.0, max_requests=None):
     return dict(seconds=total_t, tokens=total_tok, requests=n, passes=passes, cores=oracle.num_threads())
 
 
+WORKLOAD_HELP = ("config2 (default, the named benchmark) | config1 | config3 | config4 | "
+                 "config5:<batch>:<selected>[:dense] (one sweep cell)")
+
+
+def make_workload(spec, dev, batch):
+    """Build a named workload and a one-line description of it."""
+    from paper_2511_22481_b200 import workloads as W
+    if spec == "config2":
+        w = W.config2_r1(dev, batch=batch)
+        text = ("config2 DeepSeek-R1-shaped decode: batch %d/GPU, 128 heads, d_qk 576, d_v 512, ctx 32768, "
+                "64-token pages shuffled, 2112 selected tokens/request (page 0 + last 512 + 24 middle pages), seed 1" % batch)
+    elif spec == "config1":
+        w = W.config1_tiny(dev)
+        text = "config1 tiny: batch 1, 16 heads, ctx 4096, identity page table, 832 selected tokens, seed 0"
+    elif spec == "config3":
+        w = W.config3_ragged(dev)
+        text = "config3 ragged: batch 128, 128 heads, ctx U[4096,65536], 1/8 of pages selected, seed 2"
+    elif spec == "config4":
+        w = W.config4_topk(dev)
+        text = "config4 token-level top-k: batch 16, 128 heads, ctx 131072, 2048 scattered tokens/request, seed 3"
+    elif spec.startswith("config5:"):
+        f = spec.split(":")
+        w = W.config5_cell(int(f[1]), int(f[2]), dev, dense_variant=(len(f) > 3 and f[3] == "dense"))
+        text = "config5 sweep cell: batch %s, %s tokens/request of ctx 65536, 128 heads" % (
+            f[1], "all 65536" if len(f) > 3 else f[2])
+    else:
+        raise SystemExit("unknown --workload %r; choose %s" % (spec, WORKLOAD_HELP))
+    return w, text
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -159,6 +189,7 @@ def main():
                     help="tc: tensor-core kernel (the product path); simt: plain-FMA bring-up kernel")
     ap.add_argument("--clones", type=int, default=6, help="KV pool copies rotated to keep L2 cold")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default="config2", help=WORKLOAD_HELP)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -188,10 +219,12 @@ def main():
     B.load()
 
     flags = B.OMNI_FLAG_SIMT if args.kernel == "simt" else 0
-    w = W.config2_r1(dev, batch=args.batch)
+    w, workload_text = make_workload(args.workload, dev, args.batch)
     # keep L2 cold: rotate over independent copies of the pool so the bytes touched between two
     # uses of the same copy exceed L2 several times
     clones = max(2, args.clones)
+    while clones > 2 and clones * w.kv_cache.numel() * 2 > 40e9:      # keep the rotated copies within 40 GB
+        clones -= 1
     pools = [w.kv_cache] + [w.kv_cache.clone() for _ in range(clones - 1)]
     plan = B.plan_for(w, flags=flags)
     kv_bytes = w.selected_kv_bytes
@@ -267,14 +300,12 @@ def main():
     e2e_ms_total = e_begin.elapsed_time(e_end)
 
     # ---- reduce over ranks: slowest rank's time, all ranks' bytes ------------------------
-    times = torch.tensor([ms_total, e2e_ms_total], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms_total, e2e_ms_total = (float(x) for x in times.tolist())
+    from paper_2511_22481_b200 import dp
+    (ms_total, e2e_ms_total), job_bytes = dp.job_throughput([ms_total, e2e_ms_total], kv_bytes, device=dev)
     ms_per_step = ms_total / args.steps
     e2e_ms_per_step = e2e_ms_total / e2e_steps
-    value = world * kv_bytes / (ms_per_step * 1e-3) / 1e9
-    e2e_value = world * kv_bytes / (e2e_ms_per_step * 1e-3) / 1e9
+    value = job_bytes / (ms_per_step * 1e-3) / 1e9
+    e2e_value = job_bytes / (e2e_ms_per_step * 1e-3) / 1e9
 
     if rank == 0:
         peaks = _peaks()
@@ -288,9 +319,7 @@ def main():
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": round(ms_per_step, 6), "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": "config2 DeepSeek-R1-shaped decode: batch 32/GPU, 128 heads, d_qk 576, "
-                                   "d_v 512, ctx 32768, 64-token pages shuffled, 2112 selected tokens/request "
-                                   "(page 0 + last 512 + 24 middle pages), seed 1",
+            "config": {"workload": workload_text,
                        "selected_tokens_per_gpu": w.selected_tokens, "kv_bytes_per_step_per_gpu": kv_bytes,
                        "splits": plan.splits, "kernel": args.kernel,
                        "l2": "cold: %d pool copies rotated (%.0f MB touched per cycle vs %.0f MB L2)"
@@ -337,7 +366,7 @@ def reference_arm(args):
 
     # inputs of the same workload; a reduced pool is enough because only selected rows are read
     dev = "cuda" if torch.cuda.is_available() else "cpu"
-    w = W.config2_r1(dev)
+    w, _ = make_workload(args.workload, dev, args.batch)
     per_step = max(2.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
     times, tokens = [], 0
     for i in range(args.warmup + args.steps):

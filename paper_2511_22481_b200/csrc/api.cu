@@ -68,9 +68,10 @@ int units_per_request(const omni_mla_desc_t *d)
     return (d->num_heads + kTcHeads - 1) / kTcHeads;
 }
 
-// Pick the number of split-KV partitions per request: the kernel's CTAs are laid out in
-// waves over the SMs, each CTA walking ceil(granules / S) 64-token granules, so minimise
-// waves * granules-per-CTA with a small charge per split for the merge.
+// Pick the number of split-KV partitions per request.  The kernel's work units run in waves over
+// the SMs; a unit costs a fixed part (set-up, first-tile latency, epilogue: about 6 tile times as
+// measured) plus one tile time per 64-token granule, and splitting at all costs about 6 more tile
+// times (partials written and merged).  Minimise waves * (granules per unit + 6) + merge.
 int choose_splits(const omni_mla_desc_t *d, int sm_count)
 {
     if (d->num_splits >= 1) return d->num_splits;
@@ -84,7 +85,7 @@ int choose_splits(const omni_mla_desc_t *d, int sm_count)
     for (int s = 1; s <= kMaxSplits && s <= granules; ++s) {
         const long waves = (units * s + sm_count - 1) / sm_count;
         const long per = (granules + s - 1) / s;
-        const long cost = waves * (per * 8 + 6) + (s > 1 ? 8 + s : 0);
+        const long cost = waves * (per + 6) + (s > 1 ? 6 : 0);
         if (best_cost < 0 || cost < best_cost) {
             best_cost = cost;
             best = s;
