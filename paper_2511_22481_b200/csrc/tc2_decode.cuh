@@ -25,7 +25,8 @@
 // issues one every 25-64 clocks).  Completion is broadcast to both CTAs with multicast commits.
 //
 // Warps per CTA: 0 K-role producer, 1 MMA issuer (CTA 0 only) + tensor-memory owner,
-// 2-5 softmax / epilogue, 6 V-role producer, 7 L2 prefetcher (CTA 0 only): shared memory holds
+// 2-5 and 8-11 softmax / epilogue (two warps per tensor-memory lane quarter, 16 of a tile's 64
+// tokens per thread), 6 V-role producer, 7 L2 prefetcher (CTA 0 only): shared memory holds
 // only two tiles, about one HBM latency of work, so whole pages are pulled into L2 a few tiles
 // ahead and the shared-memory refills then hit L2.
 //
@@ -44,7 +45,7 @@
 namespace omni {
 
 constexpr int kC2Tile = 64;                              // tokens per tile of the pair
-constexpr int kC2Threads = 256;
+constexpr int kC2Threads = 384;
 constexpr int kPrefetchAhead = 5;                         // tiles the L2 prefetch runs ahead of Q K^T
 constexpr int kC2KBytes = kPanels * 32 * 128;            // K role: 9 panels x [32 tokens x 128 B]
 constexpr int kC2KPanel = 32 * 128;
@@ -54,8 +55,8 @@ constexpr int kC2SmemK = kC2SmemQ + kTileBytes;          // 2 stages
 constexpr int kC2SmemV = kC2SmemK + 2 * kC2KBytes;       // 2 stages
 constexpr int kC2SmemP = kC2SmemV + 2 * kC2VBytes;       // 2 buffers x [64 heads x 128 B]
 constexpr int kC2SmemCtl = kC2SmemP + 2 * kPanelBytes;
-constexpr int kC2SmemCtlBytes = 2048;
-constexpr int kC2SmemBytes = kC2SmemCtl + kC2SmemCtlBytes + 1024;
+constexpr int kC2SmemCtlBytes = 3072;
+constexpr int kC2SmemBytes = kC2SmemCtl + kC2SmemCtlBytes;   // no alignment slack: the base is checked at run time
 constexpr uint32_t kC2ColS = 256;
 constexpr int kMaskRing = 4;
 
@@ -71,7 +72,7 @@ struct C2Control {
     uint64_t x_bar;                      // softmax threads: row-maximum exchange
     uint64_t exit_bar;                   // both CTAs of the pair are done with tensor memory
     uint64_t valid_mask[kMaskRing];      // per tile: validity of its 64 tokens
-    float xchg[2][2][64];                // [tile parity][token half][head row]
+    float xchg[2][4][64];                // [tile parity][token quarter][head row]
     uint32_t tmem_base;
     uint32_t abort;
 };
@@ -172,7 +173,12 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
                   const __grid_constant__ CUtensorMap kv_tile_map, DecodeParams p)
 {
     extern __shared__ uint8_t smem_raw[];
-    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t *smem = smem_raw;
+    if (smem_u32(smem_raw) & 1023u) {
+        // the swizzled operand layouts need a 1024-byte aligned base; never seen otherwise, but say so
+        if (threadIdx.x == 0) flag_status(p.status, OMNI_DEV_TIMEOUT);
+        return;
+    }
     C2Control *ctl = reinterpret_cast<C2Control *>(smem + kC2SmemCtl);
     const uint32_t smem_base = smem_u32(smem);
     const uint32_t rank = cluster_rank();
@@ -221,11 +227,11 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
             mbar_init(&ctl->k_empty[i], 1);
             mbar_init(&ctl->v_full[i], 1);
             mbar_init(&ctl->s_full[i], 1);
-            mbar_init(&ctl->s_empty[i], 8);      // one arrival per softmax warp of either CTA
-            mbar_init(&ctl->p_full[i], 8);
+            mbar_init(&ctl->s_empty[i], 16);     // one arrival per softmax warp of either CTA
+            mbar_init(&ctl->p_full[i], 16);
             mbar_init(&ctl->pv_done[i], 1);
         }
-        mbar_init(&ctl->x_bar, 128);
+        mbar_init(&ctl->x_bar, 256);
         mbar_init(&ctl->exit_bar, 2);
         ctl->abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -513,14 +519,21 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         __syncwarp();
     } else {
         // =========================== softmax + epilogue =================================
+        // Eight warps (2-5 and 8-11): two per tensor-memory lane quarter.  A thread serves head row
+        // L % 64 (L = its tensor-memory lane), the token half L / 64 of the tile and, within that
+        // half, the 16 tokens picked by `sub` (0 for warps 2-5, 1 for warps 8-11); of O it serves
+        // value columns 256 * (L / 64) + 128 * sub + [0, 128).  The four threads of a row exchange
+        // their partial row maximum through shared memory.
         const int quarter = warp & 3;
+        const int sub = warp >= 8 ? 1 : 0;
         const int row = (quarter & 1) * 32 + lane;          // head row within this CTA
         const int half = quarter >> 1;                      // token half of S / column half of O
+        const int part = half * 2 + sub;                    // which quarter of the tile's tokens
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-        const uint32_t s_empty_leader[2] = {map_to_rank(smem_u32(&ctl->s_empty[0]), 0),
-                                            map_to_rank(smem_u32(&ctl->s_empty[1]), 0)};
-        const uint32_t p_full_leader[2] = {map_to_rank(smem_u32(&ctl->p_full[0]), 0),
-                                           map_to_rank(smem_u32(&ctl->p_full[1]), 0)};
+        const uint32_t s_empty_leader0 = map_to_rank(smem_u32(&ctl->s_empty[0]), 0);
+        const uint32_t s_empty_leader1 = map_to_rank(smem_u32(&ctl->s_empty[1]), 0);
+        const uint32_t p_full_leader0 = map_to_rank(smem_u32(&ctl->p_full[0]), 0);
+        const uint32_t p_full_leader1 = map_to_rank(smem_u32(&ctl->p_full[1]), 0);
         float m_ref = -INFINITY, l = 0.f;
         bool ok = true;
         for (int i = 0; i < tiles; ++i) {
@@ -531,37 +544,38 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
                 break;
             }
             tc_fence_after();
-            uint32_t sv[32];
-            tc_ld32(tmem + lane_base + kC2ColS + 32 * buf, sv);
+            uint32_t sv[16];
+            tc_ld16(tmem + lane_base + kC2ColS + 32 * buf + 16 * sub, sv);
             tc_wait_ld();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(s_empty_leader[buf]);
-            const uint32_t valid = (uint32_t)(ctl->valid_mask[i % kMaskRing] >> (32 * half));
-            float x[32];
+            if (lane == 0) mbar_arrive_cluster(buf ? s_empty_leader1 : s_empty_leader0);
+            const uint32_t valid = (uint32_t)(ctl->valid_mask[i % kMaskRing] >> (16 * part)) & 0xffffu;
+            float x[16];
             float mt = -INFINITY;
-            if (valid == 0xffffffffu) {
+            if (valid == 0xffffu) {
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
+                for (int j = 0; j < 16; ++j) {
                     x[j] = __uint_as_float(sv[j]) * p.scale_log2;
                     mt = fmaxf(mt, x[j]);
                 }
             } else {
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
+                for (int j = 0; j < 16; ++j) {
                     x[j] = ((valid >> j) & 1u) ? __uint_as_float(sv[j]) * p.scale_log2 : -INFINITY;
                     mt = fmaxf(mt, x[j]);
                 }
             }
-            // the other token half of this row lives in the warp two quarters away
-            ctl->xchg[i & 1][half][row] = mt;
+            ctl->xchg[i & 1][part][row] = mt;
             mbar_arrive(&ctl->x_bar);
             ok = mbar_wait(&ctl->x_bar, i & 1);
             if (!__all_sync(0xffffffffu, ok)) {
                 ok = false;
                 break;
             }
-            mt = fmaxf(mt, ctl->xchg[i & 1][half ^ 1][row]);
+            mt = fmaxf(fmaxf(ctl->xchg[i & 1][0][row], ctl->xchg[i & 1][1][row]),
+                       fmaxf(ctl->xchg[i & 1][2][row], ctl->xchg[i & 1][3][row]));
+            // move the reference only when the tile maximum leaves the window above it
             float factor = 1.f;
             bool moved = false;
             if (mt > m_ref + kRescaleThreshold || (m_ref == -INFINITY && mt > -INFINITY)) {
@@ -571,9 +585,9 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
             }
             const float mr = (m_ref == -INFINITY) ? 0.f : m_ref;
             float sum = 0.f;
-            uint32_t pk[16];
+            uint32_t pk[8];
 #pragma unroll
-            for (int j = 0; j < 32; j += 2) {
+            for (int j = 0; j < 16; j += 2) {
                 const float e0 = exp2f(x[j] - mr), e1 = exp2f(x[j + 1] - mr);
                 sum += e0 + e1;
                 pk[j >> 1] = pack_bf16(e0, e1);
@@ -595,36 +609,36 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
                 }
                 tc_fence_after();
 #pragma unroll 1
-                for (int c = 0; c < 256; c += 32) {
+                for (int c = 0; c < 128; c += 32) {
                     uint32_t ov[32];
-                    tc_ld32(tmem + lane_base + kColO + c, ov);
+                    tc_ld32(tmem + lane_base + kColO + 128 * sub + c, ov);
                     tc_wait_ld();
 #pragma unroll
                     for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * factor);
-                    tc_st32(tmem + lane_base + kColO + c, ov);
+                    tc_st32(tmem + lane_base + kColO + 128 * sub + c, ov);
                 }
                 tc_wait_st();
             }
-            // P row half: 32 tokens x bf16 = 64 B = four 16-byte chunks, chunk c stored at c ^ (row % 8)
+            // P row quarter: 16 tokens x bf16 = two 16-byte chunks, chunk c stored at c ^ (row % 8)
             uint8_t *p_row = smem + kC2SmemP + buf * kPanelBytes + row * 128;
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const int chunk = (half * 4 + c) ^ (row & 7);
+            for (int c = 0; c < 2; ++c) {
+                const int chunk = (part * 2 + c) ^ (row & 7);
                 *reinterpret_cast<uint4 *>(p_row + chunk * 16) =
                     make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
             }
             fence_async_smem();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(p_full_leader[buf]);
+            if (lane == 0) mbar_arrive_cluster(buf ? p_full_leader1 : p_full_leader0);
         }
         if (ok) {
             ok = mbar_wait(&ctl->pv_done[(tiles - 1) & 1], ((tiles - 1) >> 1) & 1);
             ok = __all_sync(0xffffffffu, ok);
         }
         if (ok) {
-            // total row sum: add the other token half's partial sum
-            ctl->xchg[tiles & 1][half][row] = l;
+            // total row sum: add the partial sums of the row's other three threads
+            ctl->xchg[tiles & 1][part][row] = l;
             mbar_arrive(&ctl->x_bar);
             ok = mbar_wait(&ctl->x_bar, tiles & 1);
             ok = __all_sync(0xffffffffu, ok);
@@ -635,19 +649,20 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
             // by 16 B so that the 32 rows a warp writes at once fall in different banks) and leave
             // as one bulk copy per row: full-line writes instead of scattered 16-byte stores.
             tc_fence_after();
-            const float lt = l + ctl->xchg[tiles & 1][half ^ 1][row];
+            const float lt = (ctl->xchg[tiles & 1][0][row] + ctl->xchg[tiles & 1][1][row]) +
+                             (ctl->xchg[tiles & 1][2][row] + ctl->xchg[tiles & 1][3][row]);
             const float inv = lt > 0.f ? 1.f / lt : 0.f;
             const int h = h0 + row;
             const bool store = h < p.heads;
             const bool final_out = p.splits == 1;
             const size_t u = final_out ? ((size_t)b * p.heads + h) : (((size_t)b * p.splits + s) * p.heads + h);
             const uint32_t row_bytes = final_out ? kDv * 2 : kDv * 4, pitch = row_bytes + 16;
-            uint8_t *stage_row = smem + (size_t)row * pitch + half * (row_bytes / 2);
+            uint8_t *stage_row = smem + (size_t)row * pitch + part * (row_bytes / 4);
 #pragma unroll 1
-            for (int c = 0; c < 256; c += 32) {
+            for (int c = 0; c < 128; c += 32) {
                 uint32_t ov[32];
                 __syncwarp();
-                tc_ld32(tmem + lane_base + kColO + c, ov);
+                tc_ld32(tmem + lane_base + kColO + 128 * sub + c, ov);
                 tc_wait_ld();
                 if (final_out) {
                     uint4 *o = reinterpret_cast<uint4 *>(stage_row + c * 2);
@@ -668,19 +683,19 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
                                            __uint_as_float(ov[4 * j + 2]) * inv, __uint_as_float(ov[4 * j + 3]) * inv);
                 }
             }
-            if (store && half == 0) {
+            if (store && part == 0) {
                 const float lse = lt > 0.f ? (m_ref + log2f(lt)) * kLn2 : -INFINITY;
                 if (final_out)
                     p.lse[u] = lse;
                 else
                     p.part_lse[u] = lse;
             }
-            // both halves of every row staged -> the thread that owns the first half sends the row
+            // all four quarters of every row staged -> the thread that owns the first quarter sends the row
             fence_async_smem();
             mbar_arrive(&ctl->x_bar);
             ok = mbar_wait(&ctl->x_bar, (tiles + 1) & 1);
             ok = __all_sync(0xffffffffu, ok);
-            if (ok && store && half == 0) {
+            if (ok && store && part == 0) {
                 uint8_t *dst = final_out ? reinterpret_cast<uint8_t *>(p.out + u * kDv)
                                          : reinterpret_cast<uint8_t *>(p.part_out + u * kDv);
                 asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst),
