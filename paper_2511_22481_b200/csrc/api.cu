@@ -117,9 +117,22 @@ omni_status_t launch_combine(int batch, int heads, int max_splits, const float *
         cudaFuncSetAttribute(combine_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
         carveout_set = true;
     }
-    combine_kernel<<<batch * heads, 128, 0, stream>>>(part_out, part_lse, num_splits, max_splits,
-                                                      heads, static_cast<__nv_bfloat16 *>(out), lse);
-    return cudaPeekAtLastError() == cudaSuccess ? OMNI_OK : OMNI_ERR_CUDA;
+    // Programmatic dependent launch: the merge blocks may become resident while the decode kernel
+    // is still running and wait (griddepcontrol.wait) until it has completed and its writes are
+    // visible, which removes most of the launch gap between the two kernels.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(batch * heads));
+    cfg.blockDim = dim3(128);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, combine_kernel, part_out, part_lse, num_splits, max_splits, heads,
+                              static_cast<__nv_bfloat16 *>(out), lse) == cudaSuccess
+               ? OMNI_OK
+               : OMNI_ERR_CUDA;
 }
 
 omni_status_t launch_resolve(const omni_mla_desc_t *d, const int32_t *page_table,

@@ -14,6 +14,8 @@ __global__ void __launch_bounds__(128) combine_kernel(const float *__restrict__ 
                                                       __nv_bfloat16 *__restrict__ out,
                                                       float *__restrict__ lse)
 {
+    // no-op unless launched as a programmatic dependent: then wait for the producing kernel
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int b = blockIdx.x / heads, h = blockIdx.x % heads;
     int ns = num_splits ? __ldg(num_splits + b) : max_splits;
     ns = max(0, min(ns, max_splits));

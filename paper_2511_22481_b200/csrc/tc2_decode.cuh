@@ -189,6 +189,9 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;  // warp-uniform
     const int h0 = (int)rank * kTcHeads;
 
+    // let a dependent kernel (the split merge) be scheduled as soon as resources allow; it still
+    // waits for this grid to finish before it reads anything
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     int n = __ldg(p.sel_len + b);
     bool bad_len = false;
     if (n < 0 || n > p.max_sel) {
