@@ -35,7 +35,7 @@
 //   columns   0..255  O: two N=256 accumulators; lane L, column x  <->  head row L%64,
 //                        value column 256*(L/64) + x
 //   columns 256..287  S buffer 0: lane L, column x <-> head row L%64, token 32*(L/64) + x
-//   columns 288..319  S buffer 1
+//   columns 288..319, 320..351  S buffers 1, 2 (Q K^T runs two tiles ahead of P V)
 #pragma once
 
 #include <type_traits>
@@ -65,8 +65,8 @@ struct C2Control {
     uint64_t k_full[2];
     uint64_t k_empty[2];
     uint64_t v_full[2];
-    uint64_t s_full[2];
-    uint64_t s_empty[2];
+    uint64_t s_full[3];
+    uint64_t s_empty[3];
     uint64_t p_full[2];
     uint64_t pv_done[2];                 // P V of a tile retired: frees its V stage and its P buffer
     uint64_t x_bar;                      // softmax threads: row-maximum exchange
@@ -229,10 +229,12 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
             mbar_init(&ctl->k_full[i], 1);
             mbar_init(&ctl->k_empty[i], 1);
             mbar_init(&ctl->v_full[i], 1);
-            mbar_init(&ctl->s_full[i], 1);
-            mbar_init(&ctl->s_empty[i], 16);     // one arrival per softmax warp of either CTA
             mbar_init(&ctl->p_full[i], 16);
             mbar_init(&ctl->pv_done[i], 1);
+        }
+        for (int i = 0; i < 3; ++i) {
+            mbar_init(&ctl->s_full[i], 1);
+            mbar_init(&ctl->s_empty[i], 16);     // one arrival per softmax warp of either CTA
         }
         mbar_init(&ctl->x_bar, 256);
         mbar_init(&ctl->exit_bar, 2);
@@ -451,17 +453,17 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
             // The buffer parity is a compile-time constant of each issue routine (the tile loop is
             // unrolled by two), so every operand of an MMA is a loop-invariant uniform value.
             // S(t) = Q K(t)^T: 36 k-steps, Q panel c (8 KiB apart) against K panel c (4 KiB apart)
-            auto issue_qk = [&](auto par_tag) {
-                constexpr int par = decltype(par_tag)::value;
-                const uint32_t d = tmem_u + kC2ColS + 32 * par;
-                const uint32_t kb = k_lo + ((par * kC2KBytes) >> 4);
+            auto issue_qk = [&](auto kpar_tag, auto sbuf_tag) {
+                constexpr int kpar = decltype(kpar_tag)::value, sbuf = decltype(sbuf_tag)::value;
+                const uint32_t d = tmem_u + kC2ColS + 32 * sbuf;
+                const uint32_t kb = k_lo + ((kpar * kC2KBytes) >> 4);
                 tc_mma_pair_elect<false>(d, q_lo, kmaj_hi, kb, kmaj_hi, idesc_qk);
 #pragma unroll
                 for (int kk = 1; kk < kDqk / 16; ++kk)
                     tc_mma_pair_elect<true>(d, q_lo + (((kk >> 2) * kPanelBytes + (kk & 3) * 32) >> 4), kmaj_hi,
                                             kb + (((kk >> 2) * kC2KPanel + (kk & 3) * 32) >> 4), kmaj_hi, idesc_qk);
-                tc_commit_pair_elect(&ctl->k_empty[par]);
-                tc_commit_pair_elect(&ctl->s_full[par]);
+                tc_commit_pair_elect(&ctl->k_empty[kpar]);
+                tc_commit_pair_elect(&ctl->s_full[sbuf]);
             };
             // O += P(t) V(t): 4 k-steps of 16 tokens, two N=256 instructions each
             auto issue_pv = [&](auto par_tag, bool first) {
@@ -483,36 +485,47 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
                 }
                 tc_commit_pair_elect(&ctl->pv_done[par]);
             };
-            // one tile: Q K^T of the NEXT tile first (its K was requested two tiles ago, so the wait
-            // is normally already satisfied), then P V of this tile
-            auto step = [&](auto par_tag, int i) -> bool {
+            // Q K^T runs two tiles ahead of P V (three S buffers), so the chain S ready -> softmax ->
+            // P -> P V of a tile has two tile times to complete before the tensor pipe needs it.
+            // S(t) lives in buffer t % 3, K(t) in stage t & 1.
+            auto qk_tile = [&](auto kpar_tag, auto sbuf_tag, int t) -> bool {
+                constexpr int kpar = decltype(kpar_tag)::value, sbuf = decltype(sbuf_tag)::value;
+                bool good = mbar_wait(&ctl->k_full[kpar], (t >> 1) & 1) &&
+                            (t < 3 || mbar_wait(&ctl->s_empty[sbuf], ((t / 3) - 1) & 1));
+                good = __all_sync(0xffffffffu, good);
+                if (!good) return false;
+                tc_fence_after();
+                issue_qk(kpar_tag, sbuf_tag);
+                return true;
+            };
+            auto pv_tile = [&](auto par_tag, int i) -> bool {
                 constexpr int par = decltype(par_tag)::value;
-                bool good = true;
-                if (i + 1 < tiles_u) {
-                    const int t = i + 1;
-                    good = mbar_wait(&ctl->k_full[par ^ 1], (t >> 1) & 1) &&
-                           (t < 2 || mbar_wait(&ctl->s_empty[par ^ 1], ((t >> 1) - 1) & 1));
-                    good = __all_sync(0xffffffffu, good);
-                    if (!good) return false;
-                    tc_fence_after();
-                    issue_qk(std::integral_constant<int, par ^ 1>{});
-                }
-                good = mbar_wait(&ctl->p_full[par], (i >> 1) & 1) && mbar_wait(&ctl->v_full[par], (i >> 1) & 1);
+                bool good = mbar_wait(&ctl->p_full[par], (i >> 1) & 1) && mbar_wait(&ctl->v_full[par], (i >> 1) & 1);
                 good = __all_sync(0xffffffffu, good);
                 if (!good) return false;
                 tc_fence_after();
                 issue_pv(par_tag, i == 0);
                 return true;
             };
-            bool ok = mbar_wait(&ctl->q_full, 0) && mbar_wait(&ctl->k_full[0], 0);
+            using I0 = std::integral_constant<int, 0>;
+            using I1 = std::integral_constant<int, 1>;
+            using I2 = std::integral_constant<int, 2>;
+            // step j of a group of six tiles: Q K^T of tile i+2 (stage i & 1, buffer (i+2) % 3), then P V of tile i
+            auto step = [&](auto kpar_tag, auto sbuf_tag, int i) -> bool {
+                if (i + 2 < tiles_u && !qk_tile(kpar_tag, sbuf_tag, i + 2)) return false;
+                return pv_tile(kpar_tag, i);
+            };
+            bool ok = mbar_wait(&ctl->q_full, 0);
             ok = __all_sync(0xffffffffu, ok);
-            if (ok) {
-                tc_fence_after();
-                issue_qk(std::integral_constant<int, 0>{});
-            }
-            for (int i = 0; ok && i < tiles_u; i += 2) {
-                ok = step(std::integral_constant<int, 0>{}, i);
-                if (ok && i + 1 < tiles_u) ok = step(std::integral_constant<int, 1>{}, i + 1);
+            if (ok) ok = qk_tile(I0{}, I0{}, 0);
+            if (ok && tiles_u > 1) ok = qk_tile(I1{}, I1{}, 1);
+            for (int i = 0; ok && i < tiles_u; i += 6) {
+                ok = step(I0{}, I2{}, i);
+                if (ok && i + 1 < tiles_u) ok = step(I1{}, I0{}, i + 1);
+                if (ok && i + 2 < tiles_u) ok = step(I0{}, I1{}, i + 2);
+                if (ok && i + 3 < tiles_u) ok = step(I1{}, I2{}, i + 3);
+                if (ok && i + 4 < tiles_u) ok = step(I0{}, I0{}, i + 4);
+                if (ok && i + 5 < tiles_u) ok = step(I1{}, I1{}, i + 5);
             }
             if (!ok && lane == 0) {
                 flag_status(p.status, OMNI_DEV_TIMEOUT);
@@ -533,26 +546,25 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         const int half = quarter >> 1;                      // token half of S / column half of O
         const int part = half * 2 + sub;                    // which quarter of the tile's tokens
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-        const uint32_t s_empty_leader0 = map_to_rank(smem_u32(&ctl->s_empty[0]), 0);
-        const uint32_t s_empty_leader1 = map_to_rank(smem_u32(&ctl->s_empty[1]), 0);
+        const uint32_t s_empty_leader = map_to_rank(smem_u32(&ctl->s_empty[0]), 0);   // [1], [2] follow at +8, +16
         const uint32_t p_full_leader0 = map_to_rank(smem_u32(&ctl->p_full[0]), 0);
         const uint32_t p_full_leader1 = map_to_rank(smem_u32(&ctl->p_full[1]), 0);
         float m_ref = -INFINITY, l = 0.f;
         bool ok = true;
         for (int i = 0; i < tiles; ++i) {
-            const int buf = i & 1;
-            ok = mbar_wait(&ctl->s_full[buf], (i >> 1) & 1);
+            const int buf = i & 1, sbuf = i % 3;
+            ok = mbar_wait(&ctl->s_full[sbuf], (i / 3) & 1);
             if (!__all_sync(0xffffffffu, ok)) {
                 ok = false;
                 break;
             }
             tc_fence_after();
             uint32_t sv[16];
-            tc_ld16(tmem + lane_base + kC2ColS + 32 * buf + 16 * sub, sv);
+            tc_ld16(tmem + lane_base + kC2ColS + 32 * sbuf + 16 * sub, sv);
             tc_wait_ld();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(buf ? s_empty_leader1 : s_empty_leader0);
+            if (lane == 0) mbar_arrive_cluster(s_empty_leader + 8 * sbuf);
             const uint32_t valid = (uint32_t)(ctl->valid_mask[i % kMaskRing] >> (16 * part)) & 0xffffu;
             float x[16];
             float mt = -INFINITY;
@@ -649,8 +661,8 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         if (ok) {
             // The 64 output rows of this CTA are one contiguous block of global memory.  They are
             // staged in shared memory (all operand buffers are dead by now; the row pitch is padded
-            // by 16 B so that the 32 rows a warp writes at once fall in different banks) and leave
-            // as one bulk copy per row: full-line writes instead of scattered 16-byte stores.
+            // by 16 B so that the 32 rows a warp writes at once fall in different banks) and then
+            // written out with fully coalesced stores instead of scattered 16-byte ones.
             tc_fence_after();
             const float lt = (ctl->xchg[tiles & 1][0][row] + ctl->xchg[tiles & 1][1][row]) +
                              (ctl->xchg[tiles & 1][2][row] + ctl->xchg[tiles & 1][3][row]);
@@ -693,19 +705,23 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
                 else
                     p.part_lse[u] = lse;
             }
-            // all four quarters of every row staged -> the thread that owns the first quarter sends the row
-            fence_async_smem();
+            // all rows staged -> the 256 threads copy the block out in 16-byte pieces, consecutive
+            // threads to consecutive addresses (one bulk copy per row would cost 64 copy-engine
+            // instructions, ~3 us at the engine's instruction rate)
             mbar_arrive(&ctl->x_bar);
             ok = mbar_wait(&ctl->x_bar, (tiles + 1) & 1);
             ok = __all_sync(0xffffffffu, ok);
-            if (ok && store && part == 0) {
-                uint8_t *dst = final_out ? reinterpret_cast<uint8_t *>(p.out + u * kDv)
-                                         : reinterpret_cast<uint8_t *>(p.part_out + u * kDv);
-                asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst),
-                             "r"(smem_u32(smem + (size_t)row * pitch)), "r"(row_bytes)
-                             : "memory");
-                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+            if (ok) {
+                const int t = (sub * 4 + ((warp - 2) & 3)) * 32 + lane;          // 0..255
+                const int rows = min(kTcHeads, p.heads - h0);
+                const size_t u0 = final_out ? ((size_t)b * p.heads + h0) : (((size_t)b * p.splits + s) * p.heads + h0);
+                uint8_t *dst = final_out ? reinterpret_cast<uint8_t *>(p.out + u0 * kDv)
+                                         : reinterpret_cast<uint8_t *>(p.part_out + u0 * kDv);
+                const uint32_t total = (uint32_t)rows * row_bytes;
+                for (uint32_t off = (uint32_t)t * 16; off < total; off += 256 * 16) {
+                    const uint32_t r = off / row_bytes, c = off % row_bytes;
+                    *reinterpret_cast<uint4 *>(dst + off) = *reinterpret_cast<const uint4 *>(smem + (size_t)r * pitch + c);
+                }
             }
         }
         if (!ok && lane == 0) {
