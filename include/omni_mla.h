@@ -47,10 +47,16 @@ typedef enum {
 /* bits OR-ed into *device_status by kernels */
 #define OMNI_DEV_BAD_INDEX 1
 #define OMNI_DEV_TIMEOUT 2
+/* set together with OMNI_DEV_TIMEOUT by the paired-CTA kernel: whose wait ran out (diagnosis) */
+#define OMNI_DEV_ROLE_PRODUCER_K 0x100
+#define OMNI_DEV_ROLE_PRODUCER_V 0x200
+#define OMNI_DEV_ROLE_MMA 0x400
+#define OMNI_DEV_ROLE_SOFTMAX 0x800
 
 /* descriptor flags */
 #define OMNI_FLAG_VALIDATE 1  /* run the index validation kernel before the decode kernel  */
 #define OMNI_FLAG_SIMT 2      /* use the plain-FMA bring-up kernel instead of tensor cores */
+#define OMNI_FLAG_FUSED_MERGE 4 /* paired-CTA kernel merges the split-KV partials itself (one launch) */
 
 /* Plain-data problem descriptor; copied at call time. */
 typedef struct {
@@ -81,9 +87,10 @@ int32_t omni_sparse_mla_num_splits(const omni_mla_desc_t *desc);
 
 /*
  * Bytes of device workspace omni_sparse_mla_decode needs for this descriptor: room for the
- * fp32 partial outputs and partial log-sum-exps of every (request, split).  Returns 0 on a
- * bad descriptor.  The workspace must be 256-byte aligned; its contents need no
- * initialisation and are overwritten.
+ * fp32 partial outputs and partial log-sum-exps of every (request, split) and for the
+ * arrival counters of the in-kernel merge.  Returns 0 on a bad descriptor.  The workspace
+ * must be 256-byte aligned; its contents need no initialisation (the call clears what it
+ * needs cleared, on `stream`) and are overwritten.
  */
 size_t omni_sparse_mla_workspace_bytes(const omni_mla_desc_t *desc);
 

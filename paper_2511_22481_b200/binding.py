@@ -21,6 +21,7 @@ OMNI_DEV_BAD_INDEX = 1
 OMNI_DEV_TIMEOUT = 2
 OMNI_FLAG_VALIDATE = 1
 OMNI_FLAG_SIMT = 2
+OMNI_FLAG_FUSED_MERGE = 4
 
 EXPORTS = (
     "omni_version", "omni_status_string", "omni_sparse_mla_num_splits",

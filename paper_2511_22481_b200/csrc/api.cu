@@ -106,6 +106,25 @@ size_t part_lse_bytes(const omni_mla_desc_t *d, int splits)
     return align_up((size_t)d->batch * splits * d->num_heads * sizeof(float), 256);
 }
 
+// Arrival counters of the in-kernel merge: one per (request, head group of 64).
+size_t counter_bytes(const omni_mla_desc_t *d)
+{
+    return align_up((size_t)d->batch * ((d->num_heads + kTcHeads - 1) / kTcHeads) * sizeof(int32_t), 256);
+}
+
+size_t workspace_need(const omni_mla_desc_t *d, int splits)
+{
+    return part_out_bytes(d, splits) + part_lse_bytes(d, splits) + counter_bytes(d);
+}
+
+// On request the paired-CTA kernel merges the splits itself (the last CTA to finish a request's
+// head half does it); by default a second, programmatically dependent kernel spreads the merge
+// over all SMs, which is faster when every split of a batch finishes at about the same time.
+bool merge_in_kernel(const omni_mla_desc_t *d)
+{
+    return use_pair_kernel(d) && (d->flags & OMNI_FLAG_FUSED_MERGE);
+}
+
 omni_status_t launch_combine(int batch, int heads, int max_splits, const float *part_out,
                              const float *part_lse, const int32_t *num_splits, void *out,
                              float *lse, cudaStream_t stream)
@@ -186,8 +205,7 @@ int32_t omni_sparse_mla_num_splits(const omni_mla_desc_t *desc)
 size_t omni_sparse_mla_workspace_bytes(const omni_mla_desc_t *desc)
 {
     if (!desc_ok(desc)) return 0;
-    const int s = choose_splits(desc, device_info().sm_count);
-    return part_out_bytes(desc, s) + part_lse_bytes(desc, s) + 256;
+    return workspace_need(desc, choose_splits(desc, device_info().sm_count));
 }
 
 omni_status_t omni_sparse_mla_decode(const omni_mla_desc_t *desc, const void *q,
@@ -206,7 +224,7 @@ omni_status_t omni_sparse_mla_decode(const omni_mla_desc_t *desc, const void *q,
     if (!dev.ok) return OMNI_ERR_CUDA;
     if (dev.cc_major != 10) return OMNI_ERR_ARCH;
     const int splits = choose_splits(desc, dev.sm_count);
-    const size_t need = part_out_bytes(desc, splits) + part_lse_bytes(desc, splits) + 256;
+    const size_t need = workspace_need(desc, splits);
     if (splits > 1) {
         if (!workspace) return OMNI_ERR_NULL;
         if (!aligned(workspace, 256)) return OMNI_ERR_ALIGN;
@@ -231,6 +249,12 @@ omni_status_t omni_sparse_mla_decode(const omni_mla_desc_t *desc, const void *q,
     p.part_lse = splits > 1 ? reinterpret_cast<float *>(static_cast<char *>(workspace) + part_out_bytes(desc, splits))
                             : nullptr;
     p.status = device_status;
+    p.counters = nullptr;
+    if (splits > 1 && merge_in_kernel(desc)) {
+        p.counters = reinterpret_cast<int32_t *>(static_cast<char *>(workspace) + part_out_bytes(desc, splits) +
+                                                 part_lse_bytes(desc, splits));
+        if (cudaMemsetAsync(p.counters, 0, counter_bytes(desc), stream) != cudaSuccess) return OMNI_ERR_CUDA;
+    }
     p.num_pages = desc->num_pages;
     p.batch = desc->batch;
     p.heads = desc->num_heads;
@@ -249,7 +273,7 @@ omni_status_t omni_sparse_mla_decode(const omni_mla_desc_t *desc, const void *q,
         if (st != OMNI_OK) return st;
     }
     if (g_profile_before && g_profile_after) cudaEventRecord(g_profile_after, stream);
-    if (splits > 1)
+    if (splits > 1 && p.counters == nullptr)
         return launch_combine(desc->batch, desc->num_heads, splits, p.part_out, p.part_lse, nullptr,
                               out, lse, stream);
     return OMNI_OK;
@@ -288,6 +312,21 @@ omni_status_t omni_sparse_mla_resolve_rows(const omni_mla_desc_t *desc,
     return launch_resolve(desc, page_table, sel_idx, sel_len, rows, nullptr,
                           static_cast<cudaStream_t>(stream));
 }
+
+#ifdef OMNI_TRACE
+// development builds only: copies the timeline records of the last launches to the host
+int omni_trace_read(void *host, size_t bytes)
+{
+    if (bytes > sizeof(unsigned long long) * 2 * kTraceWarps * kTraceEvents) return 1;
+    return cudaMemcpyFromSymbol(host, g_trace, bytes) == cudaSuccess ? 0 : 2;
+}
+int omni_trace_clear(void)
+{
+    void *ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_trace) != cudaSuccess) return 2;
+    return cudaMemset(ptr, 0, sizeof(unsigned long long) * 2 * kTraceWarps * kTraceEvents) == cudaSuccess ? 0 : 2;
+}
+#endif
 
 size_t omni_sparse_mla_host_staging_bytes(const omni_mla_desc_t *desc)
 {

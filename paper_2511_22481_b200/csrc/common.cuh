@@ -28,6 +28,8 @@ struct DecodeParams {
     float *part_out;               // [B, S, H, 512]  (S > 1 only)
     float *part_lse;               // [B, S, H]
     int32_t *status;               // may be null
+    int32_t *counters;             // [B, head groups] arrivals per merge unit, zeroed before the
+                                   // launch; null: the caller merges with a kernel of its own
     int64_t num_pages;
     int32_t batch, heads, max_pages, max_sel, splits;
     float scale_log2;              // softmax_scale * log2(e)
@@ -61,5 +63,29 @@ __device__ __forceinline__ void flag_status(int32_t *status, int32_t bits)
 {
     if (status != nullptr) atomicOr(status, bits);
 }
+
+// Timeline probe of development builds (-DOMNI_TRACE; never defined in the shipped library):
+// lane 0 of every warp of the first two CTAs appends (time in ns, tile, event id) records that
+// omni_trace_read copies out.
+#ifdef OMNI_TRACE
+constexpr int kTraceWarps = 12, kTraceEvents = 1024;
+__device__ unsigned long long g_trace[2][kTraceWarps][kTraceEvents];
+__device__ __forceinline__ unsigned long long trace_time_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+#define OMNI_TRACE_DECL int trace_n = 0;
+#define OMNI_STAMP(ev, tile)                                                                        \
+    do {                                                                                            \
+        if (blockIdx.x < 2 && (threadIdx.x & 31) == 0 && trace_n < kTraceEvents)                    \
+            g_trace[blockIdx.x][threadIdx.x >> 5][trace_n++] =                                      \
+                (trace_time_ns() << 20) | ((unsigned long long)((tile) & 0xfff) << 8) | (ev);       \
+    } while (0)
+#else
+#define OMNI_TRACE_DECL
+#define OMNI_STAMP(ev, tile)
+#endif
 
 }  // namespace omni

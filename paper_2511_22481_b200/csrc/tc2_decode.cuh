@@ -36,10 +36,15 @@
 //                        value column 256*(L/64) + x
 //   columns 256..287  S buffer 0: lane L, column x <-> head row L%64, token 32*(L/64) + x
 //   columns 288..319, 320..351  S buffers 1, 2 (Q K^T runs two tiles ahead of P V)
+//
+// With more than one split per request the last CTA to finish a request's head half merges the
+// partial results itself (a counter per (request, head half) in the workspace), so a decode
+// call is one launch.
 #pragma once
 
 #include <type_traits>
 
+#include "merge.cuh"
 #include "tc_decode.cuh"
 
 namespace omni {
@@ -75,6 +80,8 @@ struct C2Control {
     float xchg[2][4][64];                // [tile parity][token quarter][head row]
     uint32_t tmem_base;
     uint32_t abort;
+    uint32_t merge_flag;
+    int32_t k_progress;                  // tiles whose K loads the producer has started (L2 prefetch pacing)
 };
 static_assert(sizeof(C2Control) <= kC2SmemCtlBytes, "control block too large");
 static_assert(kC2SmemBytes <= 232448, "shared memory budget");
@@ -188,9 +195,12 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     const int b = pair / p.splits;
     const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;  // warp-uniform
     const int h0 = (int)rank * kTcHeads;
+    const int head_rows = min(kTcHeads, p.heads - h0);
+    OMNI_TRACE_DECL
+    OMNI_STAMP(0x04, 0);
 
-    // let a dependent kernel (the split merge) be scheduled as soon as resources allow; it still
-    // waits for this grid to finish before it reads anything
+    // let a dependent kernel be scheduled as soon as resources allow; it still waits for this
+    // grid to finish before it reads anything
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     int n = __ldg(p.sel_len + b);
     bool bad_len = false;
@@ -205,9 +215,8 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     if (tiles == 0) {
         // empty split (the same decision in both CTAs of the pair): zeros and -inf, no cluster work
         if (threadIdx.x == 0 && bad_len && rank == 0) flag_status(p.status, OMNI_DEV_BAD_INDEX);
-        for (int r = warp; r < kTcHeads; r += kC2Threads / 32) {
+        for (int r = warp; r < head_rows; r += kC2Threads / 32) {
             const int h = h0 + r;
-            if (h >= p.heads) break;
             if (p.splits == 1) {
                 uint4 *o = reinterpret_cast<uint4 *>(p.out + ((size_t)b * p.heads + h) * kDv);
                 for (int i = lane; i < kDv * 2 / 16; i += 32) o[i] = make_uint4(0, 0, 0, 0);
@@ -218,6 +227,10 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
                 for (int i = lane; i < kDv / 4; i += 32) o[i] = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (lane == 0) p.part_lse[u] = -INFINITY;
             }
+        }
+        if (p.splits > 1 && p.counters != nullptr) {
+            __threadfence();
+            merge_if_last(p, b, (int)rank, 2, h0, head_rows, reinterpret_cast<float *>(smem), &ctl->merge_flag);
         }
         return;
     }
@@ -239,6 +252,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         mbar_init(&ctl->x_bar, 256);
         mbar_init(&ctl->exit_bar, 2);
         ctl->abort = 0;
+        ctl->k_progress = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -253,6 +267,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     tc_fence_after();
     const uint32_t tmem = ctl->tmem_base;
     volatile uint32_t *abort_flag = &ctl->abort;
+    OMNI_STAMP(0x01, 0);
 
     const int32_t *sel = p.sel_idx + (size_t)b * p.max_sel;
     const int32_t *pt = p.page_table + (size_t)b * p.max_pages;
@@ -273,7 +288,8 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         x.pg0 = (x.t0 >= 0 && x.t0 / kPage < p.max_pages) ? __ldg(pt + x.t0 / kPage) : -1;
         x.pg1 = (x.t1 >= 0 && x.t1 / kPage < p.max_pages) ? __ldg(pt + x.t1 / kPage) : -1;
     };
-    // row_lo / row_hi: pool rows of tokens lane and lane+32 (row 0 stands in for masked tokens);
+    // row_lo / row_hi: pool rows of tokens lane and lane+32 (a masked token repeats the row of the
+    // tile's first valid token: real cache contents, multiplied by a weight of exactly zero);
     // contig: all 64 tokens valid and in consecutive rows; contig_lo / contig_hi: the same per 32.
     auto stage_rows = [&](int tile, const TileIdx &x, int &row_lo, int &row_hi, uint64_t &mask, bool &contig,
                           bool &contig_lo, bool &contig_hi, bool &any_bad) {
@@ -283,8 +299,13 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         const int r0 = ok0 ? x.pg0 * kPage + x.t0 % kPage : -1, r1 = ok1 ? x.pg1 * kPage + x.t1 % kPage : -1;
         const uint32_t m0 = __ballot_sync(0xffffffffu, r0 >= 0), m1 = __ballot_sync(0xffffffffu, r1 >= 0);
         mask = (uint64_t)m0 | ((uint64_t)m1 << 32);
-        row_lo = r0 >= 0 ? r0 : 0;
-        row_hi = r1 >= 0 ? r1 : 0;
+        int stand_in = 0;
+        if (m0)
+            stand_in = __shfl_sync(0xffffffffu, r0, __ffs(m0) - 1);
+        else if (m1)
+            stand_in = __shfl_sync(0xffffffffu, r1, __ffs(m1) - 1);
+        row_lo = r0 >= 0 ? r0 : stand_in;
+        row_hi = r1 >= 0 ? r1 : stand_in;
         const int base_lo = __shfl_sync(0xffffffffu, row_lo, 0), base_hi = __shfl_sync(0xffffffffu, row_hi, 0);
         contig_lo = __all_sync(0xffffffffu, r0 == base_lo + lane);
         contig_hi = __all_sync(0xffffffffu, r1 == base_hi + lane);
@@ -304,16 +325,22 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         int row_lo, row_hi;
         uint64_t mask;
         bool contig, contig_lo, contig_hi;
-        stage_tokens(0, x1);
-        stage_pages(x1);
-        stage_rows(0, x1, row_lo, row_hi, mask, contig, contig_lo, contig_hi, any_bad);
-        stage_tokens(1, x1);
-        stage_pages(x1);
-        stage_tokens(2, x2);
+        {
+            // the position loads of the first three tiles go out together, then the two page-id
+            // loads that depend on them: two cache misses in a row before the first copy, not four
+            TileIdx x0;
+            stage_tokens(0, x0);
+            stage_tokens(1, x1);
+            stage_tokens(2, x2);
+            stage_pages(x0);
+            stage_pages(x1);
+            stage_rows(0, x0, row_lo, row_hi, mask, contig, contig_lo, contig_hi, any_bad);
+        }
         bool ok = true;
         for (int i = 0; ok && i < tiles; ++i) {
             const int st = i & 1;
             if (lane == 0) {
+                *const_cast<volatile int32_t *>(&ctl->k_progress) = i;
                 ctl->valid_mask[i % kMaskRing] = mask;
                 __threadfence_block();
             }
@@ -323,6 +350,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
             const uint32_t bar = map_to_rank(smem_u32(&ctl->k_full[st]), 0);
             if (lane == 0 && rank == 0) mbar_expect_tx(&ctl->k_full[st], 2 * kC2KBytes);
             __syncwarp();
+            OMNI_STAMP(0x10, i);
             const uint32_t dst = smem_base + kC2SmemK + st * kC2KBytes;
             const int own_row = rank ? row_hi : row_lo;
             if (rank ? contig_hi : contig_lo) {
@@ -344,8 +372,9 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
             stage_pages(x1);
             stage_tokens(i + 3, x2);
         }
+        if (lane == 0) *const_cast<volatile int32_t *>(&ctl->k_progress) = 0x7fffffff;
         if (!ok && lane == 0) {
-            flag_status(p.status, OMNI_DEV_TIMEOUT);
+            flag_status(p.status, OMNI_DEV_TIMEOUT | OMNI_DEV_ROLE_PRODUCER_K);
             *abort_flag = 1;
         }
         if (__any_sync(0xffffffffu, any_bad) && lane == 0 && rank == 0) flag_status(p.status, OMNI_DEV_BAD_INDEX);
@@ -357,12 +386,17 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         int row_lo, row_hi;
         uint64_t mask_unused;
         bool contig, contig_lo, contig_hi;
-        stage_tokens(0, x1);
-        stage_pages(x1);
-        stage_rows(0, x1, row_lo, row_hi, mask_unused, contig, contig_lo, contig_hi, any_bad);
-        stage_tokens(1, x1);
-        stage_pages(x1);
-        stage_tokens(2, x2);
+        {
+            // the position loads of the first three tiles go out together, then the two page-id
+            // loads that depend on them: two cache misses in a row before the first copy, not four
+            TileIdx x0;
+            stage_tokens(0, x0);
+            stage_tokens(1, x1);
+            stage_tokens(2, x2);
+            stage_pages(x0);
+            stage_pages(x1);
+            stage_rows(0, x0, row_lo, row_hi, mask_unused, contig, contig_lo, contig_hi, any_bad);
+        }
         bool ok = true;
         for (int i = 0; ok && i < tiles; ++i) {
             const int st = i & 1;
@@ -372,6 +406,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
             const uint32_t bar = map_to_rank(smem_u32(&ctl->v_full[st]), 0);
             if (lane == 0 && rank == 0) mbar_expect_tx(&ctl->v_full[st], 2 * kC2VBytes);
             __syncwarp();
+            OMNI_STAMP(0x50, i);
             const uint32_t dst = smem_base + kC2SmemV + st * kC2VBytes;
             if (contig) {
                 if (lane == 0) tma_box3d_pair(dst, &kv_v_map, bar, row_lo, 4 * (int)rank);
@@ -397,7 +432,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
             stage_tokens(i + 3, x2);
         }
         if (!ok && lane == 0) {
-            flag_status(p.status, OMNI_DEV_TIMEOUT);
+            flag_status(p.status, OMNI_DEV_TIMEOUT | OMNI_DEV_ROLE_PRODUCER_V);
             *abort_flag = 1;
         }
     } else if (warp == 7) {
@@ -420,12 +455,18 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
                 const int count = min(32, tiles - t0);
                 bool ok = true;
                 for (int k = 0; ok && k < count; ++k) {
+                    // tile i is prefetched once the K loads of tile i - kPrefetchAhead have started (a
+                    // monotonic counter, polled with a bounded number of naps)
                     const int i = t0 + k;
-                    if (i >= kPrefetchAhead + 2) {
-                        const int c = i - kPrefetchAhead;       // wait until Q K^T of tile c-2 retired
-                        ok = mbar_wait(&ctl->k_empty[c & 1], ((c >> 1) - 1) & 1);
-                        ok = __all_sync(0xffffffffu, ok) && (*abort_flag == 0);
+                    const volatile int32_t *progress = &ctl->k_progress;
+                    for (int naps = 0; *progress < i - kPrefetchAhead && *abort_flag == 0; ++naps) {
+                        if (naps > (1 << 22)) {
+                            ok = false;
+                            break;
+                        }
+                        __nanosleep(200);
                     }
+                    ok = ok && (*abort_flag == 0);
                     if (ok && lane == k && row >= 0)
                         asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(&kv_tile_map),
                                      "r"(0), "r"(row), "r"(0)
@@ -495,7 +536,9 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
                 good = __all_sync(0xffffffffu, good);
                 if (!good) return false;
                 tc_fence_after();
+                OMNI_STAMP(0x20, t);
                 issue_qk(kpar_tag, sbuf_tag);
+                OMNI_STAMP(0x28, t);
                 return true;
             };
             auto pv_tile = [&](auto par_tag, int i) -> bool {
@@ -504,7 +547,9 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
                 good = __all_sync(0xffffffffu, good);
                 if (!good) return false;
                 tc_fence_after();
+                OMNI_STAMP(0x30, i);
                 issue_pv(par_tag, i == 0);
+                OMNI_STAMP(0x38, i);
                 return true;
             };
             using I0 = std::integral_constant<int, 0>;
@@ -528,7 +573,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
                 if (ok && i + 5 < tiles_u) ok = step(I1{}, I1{}, i + 5);
             }
             if (!ok && lane == 0) {
-                flag_status(p.status, OMNI_DEV_TIMEOUT);
+                flag_status(p.status, OMNI_DEV_TIMEOUT | OMNI_DEV_ROLE_MMA);
                 *abort_flag = 1;
             }
         }
@@ -560,6 +605,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
             }
             tc_fence_after();
             uint32_t sv[16];
+            OMNI_STAMP(0x40, i);
             tc_ld16(tmem + lane_base + kC2ColS + 32 * sbuf + 16 * sub, sv);
             tc_wait_ld();
             tc_fence_before();
@@ -646,9 +692,11 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(buf ? p_full_leader1 : p_full_leader0);
+            OMNI_STAMP(0x43, i);
         }
         if (ok) {
             ok = mbar_wait(&ctl->pv_done[(tiles - 1) & 1], ((tiles - 1) >> 1) & 1);
+            OMNI_STAMP(0x48, 0);
             ok = __all_sync(0xffffffffu, ok);
         }
         if (ok) {
@@ -713,19 +761,20 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
             ok = __all_sync(0xffffffffu, ok);
             if (ok) {
                 const int t = (sub * 4 + ((warp - 2) & 3)) * 32 + lane;          // 0..255
-                const int rows = min(kTcHeads, p.heads - h0);
                 const size_t u0 = final_out ? ((size_t)b * p.heads + h0) : (((size_t)b * p.splits + s) * p.heads + h0);
                 uint8_t *dst = final_out ? reinterpret_cast<uint8_t *>(p.out + u0 * kDv)
                                          : reinterpret_cast<uint8_t *>(p.part_out + u0 * kDv);
-                const uint32_t total = (uint32_t)rows * row_bytes;
+                const uint32_t total = (uint32_t)head_rows * row_bytes;
                 for (uint32_t off = (uint32_t)t * 16; off < total; off += 256 * 16) {
                     const uint32_t r = off / row_bytes, c = off % row_bytes;
                     *reinterpret_cast<uint4 *>(dst + off) = *reinterpret_cast<const uint4 *>(smem + (size_t)r * pitch + c);
                 }
+                if (!final_out) __threadfence();       // partial results visible before this CTA is counted
+                OMNI_STAMP(0x49, 0);
             }
         }
         if (!ok && lane == 0) {
-            flag_status(p.status, OMNI_DEV_TIMEOUT);
+            flag_status(p.status, OMNI_DEV_TIMEOUT | OMNI_DEV_ROLE_SOFTMAX);
             *abort_flag = 1;
         }
     }
@@ -751,6 +800,11 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
+    // ---- split merge by whichever CTA finishes a (request, head half) last ---------------
+    OMNI_STAMP(0x02, 0);
+    if (p.splits > 1 && p.counters != nullptr)
+        merge_if_last(p, b, (int)rank, 2, h0, head_rows, reinterpret_cast<float *>(smem), &ctl->merge_flag);
+    OMNI_STAMP(0x03, 0);
 }
 
 inline omni_status_t launch_tc2_decode(const DecodeParams &p, cudaStream_t stream)

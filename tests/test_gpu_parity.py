@@ -13,7 +13,7 @@ from parity import check_workload, compare, oracle_subset, run_gpu
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
-IMPLS = {"simt": B.OMNI_FLAG_SIMT, "tc": 0}
+IMPLS = {"simt": B.OMNI_FLAG_SIMT, "tc": 0, "tc_fused_merge": B.OMNI_FLAG_FUSED_MERGE}
 
 
 @pytest.fixture(params=list(IMPLS))
@@ -132,6 +132,25 @@ def test_single_token_returns_its_row_exactly(flags):
     assert torch.equal(plan.out[0], w.kv_cache.view(-1, 576)[row, :512].expand(128, 512))
     ref_out, ref_lse, _ = oracle_subset(w)
     assert np.abs(plan.lse.cpu().numpy() - ref_lse).max() < 1e-4
+
+
+def test_rows_outside_the_selection_are_never_used(flags):
+    # every pool row that is not selected holds NaN: a kernel that pads tiles with rows of its
+    # own choosing, or reads beyond a ragged tail, poisons its output
+    rng = np.random.default_rng(49)
+    lens = [1, 3, 63, 64, 65, 100, 128, 129, 191, 300]
+    sels = [rng.permutation(12 * 64)[:n] for n in lens]
+    sels[3] = np.arange(5 * 64, 6 * 64)              # one whole page in order
+    sels[6] = np.arange(2 * 64, 4 * 64)              # two whole pages in order
+    sels[7] = np.arange(2 * 64, 4 * 64 + 1)          # two pages and one token
+    w = _custom("nan_outside", 49, 128, [12] * len(lens), sels)
+    rows = oracle.resolve_rows(w.page_table.cpu().numpy(), w.sel_idx.cpu().numpy(),
+                               w.sel_len.cpu().numpy(), 64, w.num_pages)
+    keep = torch.zeros(w.num_pages * 64, dtype=torch.bool, device=DEV)
+    keep[torch.from_numpy(rows[rows >= 0]).to(DEV)] = True
+    w.kv_cache.view(-1, 576)[~keep] = float("nan")
+    for s in (0, 1, 3):
+        check_workload(w, flags, num_splits=s, what="nan outside S=%d" % s)
 
 
 def test_out_of_range_entries_are_flagged_and_skipped(flags):
