@@ -57,6 +57,7 @@ typedef enum {
 #define OMNI_FLAG_VALIDATE 1  /* run the index validation kernel before the decode kernel  */
 #define OMNI_FLAG_SIMT 2      /* use the plain-FMA bring-up kernel instead of tensor cores */
 #define OMNI_FLAG_FUSED_MERGE 4 /* paired-CTA kernel merges the split-KV partials itself (one launch) */
+#define OMNI_FLAG_NO_CLUSTER_MERGE 8 /* never merge two splits inside a cluster of two CTA pairs */
 
 /* Plain-data problem descriptor; copied at call time. */
 typedef struct {

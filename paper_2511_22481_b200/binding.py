@@ -22,6 +22,7 @@ OMNI_DEV_TIMEOUT = 2
 OMNI_FLAG_VALIDATE = 1
 OMNI_FLAG_SIMT = 2
 OMNI_FLAG_FUSED_MERGE = 4
+OMNI_FLAG_NO_CLUSTER_MERGE = 8
 
 EXPORTS = (
     "omni_version", "omni_status_string", "omni_sparse_mla_num_splits",

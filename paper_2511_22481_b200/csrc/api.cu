@@ -250,6 +250,12 @@ omni_status_t omni_sparse_mla_decode(const omni_mla_desc_t *desc, const void *q,
                             : nullptr;
     p.status = device_status;
     p.counters = nullptr;
+    p.cluster_merge = 0;
+    // Two splits of a request can be merged inside a cluster of two CTA pairs, without partial
+    // results in global memory, as long as all those clusters are resident at once.
+    if (splits == 2 && use_pair_kernel(desc) && !(desc->flags & (OMNI_FLAG_FUSED_MERGE | OMNI_FLAG_NO_CLUSTER_MERGE)) &&
+        desc->batch <= tc2_max_merge_clusters())
+        p.cluster_merge = 1;
     if (splits > 1 && merge_in_kernel(desc)) {
         p.counters = reinterpret_cast<int32_t *>(static_cast<char *>(workspace) + part_out_bytes(desc, splits) +
                                                  part_lse_bytes(desc, splits));
@@ -273,7 +279,7 @@ omni_status_t omni_sparse_mla_decode(const omni_mla_desc_t *desc, const void *q,
         if (st != OMNI_OK) return st;
     }
     if (g_profile_before && g_profile_after) cudaEventRecord(g_profile_after, stream);
-    if (splits > 1 && p.counters == nullptr)
+    if (splits > 1 && p.counters == nullptr && !p.cluster_merge)
         return launch_combine(desc->batch, desc->num_heads, splits, p.part_out, p.part_lse, nullptr,
                               out, lse, stream);
     return OMNI_OK;
@@ -319,6 +325,11 @@ int omni_trace_read(void *host, size_t bytes)
 {
     if (bytes > sizeof(unsigned long long) * 2 * kTraceWarps * kTraceEvents) return 1;
     return cudaMemcpyFromSymbol(host, g_trace, bytes) == cudaSuccess ? 0 : 2;
+}
+int omni_span_read(void *host, size_t bytes)
+{
+    if (bytes > sizeof(unsigned long long) * 2048 * 4) return 1;
+    return cudaMemcpyFromSymbol(host, g_span, bytes) == cudaSuccess ? 0 : 2;
 }
 int omni_trace_clear(void)
 {

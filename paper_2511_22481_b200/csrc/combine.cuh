@@ -14,8 +14,10 @@ __global__ void __launch_bounds__(128) combine_kernel(const float *__restrict__ 
                                                       __nv_bfloat16 *__restrict__ out,
                                                       float *__restrict__ lse)
 {
-    // no-op unless launched as a programmatic dependent: then wait for the producing kernel
+    // no-op unless launched as a programmatic dependent: then wait for the producing kernel;
+    // the kernel that follows may be scheduled early in turn (it waits before it reads)
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int b = blockIdx.x / heads, h = blockIdx.x % heads;
     int ns = num_splits ? __ldg(num_splits + b) : max_splits;
     ns = max(0, min(ns, max_splits));

@@ -32,6 +32,7 @@ struct DecodeParams {
                                    // launch; null: the caller merges with a kernel of its own
     int64_t num_pages;
     int32_t batch, heads, max_pages, max_sel, splits;
+    int32_t cluster_merge;         // 1: two splits, merged inside a cluster of two CTA pairs
     float scale_log2;              // softmax_scale * log2(e)
 };
 
@@ -76,6 +77,11 @@ __device__ __forceinline__ unsigned long long trace_time_ns()
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
+__device__ unsigned long long g_span[2048][4];   // per CTA: entry, set-up done, last P V retired, exit
+#define OMNI_SPAN(slot)                                                                             \
+    do {                                                                                            \
+        if (threadIdx.x == 64 && blockIdx.x < 2048) g_span[blockIdx.x][slot] = trace_time_ns();     \
+    } while (0)
 #define OMNI_TRACE_DECL int trace_n = 0;
 #define OMNI_STAMP(ev, tile)                                                                        \
     do {                                                                                            \
@@ -86,6 +92,7 @@ __device__ __forceinline__ unsigned long long trace_time_ns()
 #else
 #define OMNI_TRACE_DECL
 #define OMNI_STAMP(ev, tile)
+#define OMNI_SPAN(slot)
 #endif
 
 }  // namespace omni

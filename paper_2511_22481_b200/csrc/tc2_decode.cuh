@@ -82,6 +82,8 @@ struct C2Control {
     uint32_t abort;
     uint32_t merge_flag;
     int32_t k_progress;                  // tiles whose K loads the producer has started (L2 prefetch pacing)
+    uint64_t recv_bar;                   // cluster merge: the partner's block has arrived
+    float xlse[2][64];                   // cluster merge: log-sum-exp of either split, per head row
 };
 static_assert(sizeof(C2Control) <= kC2SmemCtlBytes, "control block too large");
 static_assert(kC2SmemBytes <= 232448, "shared memory budget");
@@ -163,15 +165,112 @@ __device__ __forceinline__ void tc_mma_pair_elect(uint32_t d_tmem, uint32_t a_lo
 
 // Arrive on the barrier at this shared-memory offset in BOTH CTAs once all MMAs issued so far by
 // the elected lane have retired.
-__device__ __forceinline__ void tc_commit_pair_elect(uint64_t *bar)
+__device__ __forceinline__ void tc_commit_pair_elect(uint64_t *bar, uint16_t both)
 {
-    const uint16_t both = 3;
     asm volatile(
         "{\n\t.reg .pred q;\n\t"
         "elect.sync _|q, 0xffffffff;\n\t"
         "@q tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;\n\t}"
         ::"r"(smem_u32(bar)), "h"(both)
         : "memory");
+}
+
+// Split-KV merge inside a cluster of two pairs, i.e. the two splits of one request (cluster
+// merge).  CTA `crank` and its partner `crank ^ 2` serve the same 64 heads in the two splits.
+// Instead of writing fp32 partial results to global memory for a second kernel to read back,
+// the two exchange what the other needs through distributed shared memory:
+//   1. each tells the other the log-sum-exp of its split for every head row;
+//   2. each scales its accumulator by exp(lse_own - lse_total) / row sum, keeps the 256 value
+//      columns it will finish (split 0: columns 0..255, split 1: 256..511) and sends the other
+//      256 to the partner with one bulk shared-memory-to-shared-memory copy;
+//   3. each adds what it received to what it kept and stores its half of the final rows.
+// Called by every thread of every CTA of the cluster after the main loop; all operand buffers
+// are dead by then (the cluster barrier in step 1 is what tells a CTA that this also holds for
+// its partner, whose shared memory it writes to).
+__device__ __forceinline__ void cluster_merge_exchange(const DecodeParams &p, C2Control *ctl, uint8_t *smem,
+                                                       uint32_t tmem, int b, int s, uint32_t crank, int h0,
+                                                       int head_rows, bool active, float cm_lse, float cm_inv)
+{
+    constexpr uint32_t kSliceBytes = 256 * 4;            // half of a row's value columns, fp32
+    constexpr uint32_t kPitch = kSliceBytes + 16;        // row-per-lane 16-byte accesses do not conflict
+    constexpr uint32_t kBlockBytes = 64 * kPitch;        // 66,560
+    static_assert(3 * kBlockBytes <= kC2SmemCtl, "exchange tiles must fit below the control block");
+    uint8_t *send = smem, *keep = smem + kBlockBytes, *recv = smem + 2 * kBlockBytes;
+    const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;
+    const bool is_softmax = (warp >= 2 && warp <= 5) || warp >= 8;
+    const int quarter = warp & 3, sub = warp >= 8 ? 1 : 0;
+    const int row = (quarter & 1) * 32 + lane, part = (quarter >> 1) * 2 + sub;
+    const uint32_t partner = crank ^ 2u;
+
+    if (is_softmax && part == 0) {
+        ctl->xlse[s][row] = cm_lse;
+        const uint32_t remote = map_to_rank(smem_u32(&ctl->xlse[s][row]), partner);
+        asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(cm_lse) : "memory");
+    }
+    cluster_sync_all();
+    if (!is_softmax) return;
+
+    const float a0 = ctl->xlse[0][row], a1 = ctl->xlse[1][row];
+    const float mx = fmaxf(a0, a1);
+    float total = -INFINITY, w = 0.f;
+    if (mx > -INFINITY) {
+        total = mx + logf(exp2f((a0 - mx) * kLog2e) + exp2f((a1 - mx) * kLog2e));
+        if (cm_lse > -INFINITY) w = exp2f((cm_lse - total) * kLog2e);
+    }
+    const float f = w * cm_inv;
+    // this thread's 128 value columns are finished by split `part / 2`
+    uint8_t *tile = ((part >> 1) == s ? keep : send) + (size_t)row * kPitch + (part & 1) * 512;
+    const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+#pragma unroll 1
+    for (int q = 0; q < 4; ++q) {
+        uint32_t ov[32];
+        __syncwarp();
+        if (active) {
+            tc_ld32(tmem + lane_base + kColO + 128 * sub + q * 32, ov);
+            tc_wait_ld();
+        }
+        uint4 *o = reinterpret_cast<uint4 *>(tile + q * 128);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            // a weight of zero (empty or fully masked split) contributes exact zeros
+            o[j] = (active && f != 0.f)
+                       ? make_uint4(__float_as_uint(__uint_as_float(ov[4 * j]) * f), __float_as_uint(__uint_as_float(ov[4 * j + 1]) * f),
+                                    __float_as_uint(__uint_as_float(ov[4 * j + 2]) * f), __float_as_uint(__uint_as_float(ov[4 * j + 3]) * f))
+                       : make_uint4(0u, 0u, 0u, 0u);
+        }
+    }
+    tc_fence_before();
+    fence_async_smem();                                   // the bulk copy reads what the threads wrote
+    asm volatile("bar.sync 1, 256;" ::: "memory");         // the eight softmax warps
+    if (warp == 2 && lane == 0) {
+        mbar_expect_tx(&ctl->recv_bar, kBlockBytes);
+        const uint32_t dst = map_to_rank(smem_u32(recv), partner);
+        const uint32_t bar = map_to_rank(smem_u32(&ctl->recv_bar), partner);
+        asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(dst), "r"(smem_u32(send)), "r"(kBlockBytes), "r"(bar)
+                     : "memory");
+    }
+    bool ok = mbar_wait(&ctl->recv_bar, 0);
+    ok = __all_sync(0xffffffffu, ok);
+    if (!ok) {
+        if (lane == 0) flag_status(p.status, OMNI_DEV_TIMEOUT | OMNI_DEV_ROLE_SOFTMAX);
+        return;
+    }
+    // kept + received -> bf16, 16 output bytes (8 columns) per item, consecutive threads along a row
+    const int t = (sub * 4 + ((warp - 2) & 3)) * 32 + lane;          // 0..255
+    for (int item = t; item < head_rows * 32; item += 256) {
+        const int r = item >> 5, c = item & 31;
+        const uint4 *k4 = reinterpret_cast<const uint4 *>(keep + (size_t)r * kPitch + c * 32);
+        const uint4 *r4 = reinterpret_cast<const uint4 *>(recv + (size_t)r * kPitch + c * 32);
+        const uint4 k0 = k4[0], k1 = k4[1], r0 = r4[0], r1 = r4[1];
+        uint4 o;
+        o.x = pack_bf16(__uint_as_float(k0.x) + __uint_as_float(r0.x), __uint_as_float(k0.y) + __uint_as_float(r0.y));
+        o.y = pack_bf16(__uint_as_float(k0.z) + __uint_as_float(r0.z), __uint_as_float(k0.w) + __uint_as_float(r0.w));
+        o.z = pack_bf16(__uint_as_float(k1.x) + __uint_as_float(r1.x), __uint_as_float(k1.y) + __uint_as_float(r1.y));
+        o.w = pack_bf16(__uint_as_float(k1.z) + __uint_as_float(r1.z), __uint_as_float(k1.w) + __uint_as_float(r1.w));
+        *reinterpret_cast<uint4 *>(p.out + ((size_t)b * p.heads + h0 + r) * kDv + s * 256 + c * 8) = o;
+    }
+    if (s == 0 && part == 0 && row < head_rows) p.lse[(size_t)b * p.heads + h0 + row] = total;
 }
 
 __global__ void __launch_bounds__(kC2Threads, 1)
@@ -188,19 +287,27 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     }
     C2Control *ctl = reinterpret_cast<C2Control *>(smem + kC2SmemCtl);
     const uint32_t smem_base = smem_u32(smem);
-    const uint32_t rank = cluster_rank();
+    // A cluster is one pair, or (cluster merge) the two pairs that serve the two splits of a
+    // request.  `rank` is the CTA's place within its pair; the pair's barriers live in `leader`.
+    const uint32_t crank = cluster_rank();
+    const uint32_t rank = crank & 1u, leader = crank & ~1u, peer = crank ^ 1u;
+    const uint16_t pair_mask = (uint16_t)(3u << leader);
 
     const int pair = blockIdx.x >> 1;
-    const int s = pair % p.splits;
-    const int b = pair / p.splits;
+    const int s = p.cluster_merge ? (int)(crank >> 1) : pair % p.splits;
+    const int b = p.cluster_merge ? (int)(blockIdx.x >> 2) : pair / p.splits;
     const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;  // warp-uniform
     const int h0 = (int)rank * kTcHeads;
     const int head_rows = min(kTcHeads, p.heads - h0);
     OMNI_TRACE_DECL
     OMNI_STAMP(0x04, 0);
+    OMNI_SPAN(0);
 
-    // let a dependent kernel be scheduled as soon as resources allow; it still waits for this
-    // grid to finish before it reads anything
+    // Programmatic dependent launch, both ways.  This grid may have been scheduled while the
+    // kernel before it in the stream was still finishing: nothing in global memory is touched
+    // until that kernel has completed and its writes are visible.  And the kernel after this one
+    // may be scheduled as soon as resources allow; it waits in the same way before it reads.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     int n = __ldg(p.sel_len + b);
     bool bad_len = false;
@@ -212,9 +319,10 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     split_range(n, p.splits, s, begin, end, kC2Tile);
     const int tiles = (end - begin + kC2Tile - 1) / kC2Tile;
 
-    if (tiles == 0) {
+    const bool active = tiles > 0;
+    if (!active && bad_len && threadIdx.x == 0 && crank == 0) flag_status(p.status, OMNI_DEV_BAD_INDEX);
+    if (!active && !p.cluster_merge) {
         // empty split (the same decision in both CTAs of the pair): zeros and -inf, no cluster work
-        if (threadIdx.x == 0 && bad_len && rank == 0) flag_status(p.status, OMNI_DEV_BAD_INDEX);
         for (int r = warp; r < head_rows; r += kC2Threads / 32) {
             const int h = h0 + r;
             if (p.splits == 1) {
@@ -251,11 +359,12 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         }
         mbar_init(&ctl->x_bar, 256);
         mbar_init(&ctl->exit_bar, 2);
+        mbar_init(&ctl->recv_bar, 1);
         ctl->abort = 0;
         ctl->k_progress = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) {
+    if (warp == 1 && active) {
         asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)),
                      "r"(kTmemCols)
                      : "memory");
@@ -268,6 +377,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     const uint32_t tmem = ctl->tmem_base;
     volatile uint32_t *abort_flag = &ctl->abort;
     OMNI_STAMP(0x01, 0);
+    OMNI_SPAN(1);
 
     const int32_t *sel = p.sel_idx + (size_t)b * p.max_sel;
     const int32_t *pt = p.page_table + (size_t)b * p.max_pages;
@@ -312,10 +422,15 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         contig = contig_lo && contig_hi && base_hi == base_lo + 32;
     };
 
-    if (warp == 0) {
+    // what the cluster merge needs from the softmax warps after the main loop
+    float cm_lse = -INFINITY, cm_inv = 0.f;
+
+    if (!active) {
+        // an empty split inside a merging cluster: no pipeline, but it takes part in the exchange
+    } else if (warp == 0) {
         // =========================== K-role producer =====================================
         // This CTA's K rows are tokens [32*rank, 32*rank+32) of every tile.
-        const uint32_t q_bar = map_to_rank(smem_u32(&ctl->q_full), 0);
+        const uint32_t q_bar = map_to_rank(smem_u32(&ctl->q_full), leader);
         if (lane == 0) {
             if (rank == 0) mbar_expect_tx(&ctl->q_full, 2 * kTileBytes);
             tma_box3d_pair(smem_base + kC2SmemQ, &q_map, q_bar, b * p.heads + h0, 0);
@@ -347,7 +462,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
             if (i >= 2) ok = mbar_wait(&ctl->k_empty[st], ((i >> 1) - 1) & 1);
             ok = __all_sync(0xffffffffu, ok) && (*abort_flag == 0);
             if (!ok) break;
-            const uint32_t bar = map_to_rank(smem_u32(&ctl->k_full[st]), 0);
+            const uint32_t bar = map_to_rank(smem_u32(&ctl->k_full[st]), leader);
             if (lane == 0 && rank == 0) mbar_expect_tx(&ctl->k_full[st], 2 * kC2KBytes);
             __syncwarp();
             OMNI_STAMP(0x10, i);
@@ -403,7 +518,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
             if (i >= 2) ok = mbar_wait(&ctl->pv_done[st], ((i >> 1) - 1) & 1);
             ok = __all_sync(0xffffffffu, ok) && (*abort_flag == 0);
             if (!ok) break;
-            const uint32_t bar = map_to_rank(smem_u32(&ctl->v_full[st]), 0);
+            const uint32_t bar = map_to_rank(smem_u32(&ctl->v_full[st]), leader);
             if (lane == 0 && rank == 0) mbar_expect_tx(&ctl->v_full[st], 2 * kC2VBytes);
             __syncwarp();
             OMNI_STAMP(0x50, i);
@@ -503,8 +618,8 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
                 for (int kk = 1; kk < kDqk / 16; ++kk)
                     tc_mma_pair_elect<true>(d, q_lo + (((kk >> 2) * kPanelBytes + (kk & 3) * 32) >> 4), kmaj_hi,
                                             kb + (((kk >> 2) * kC2KPanel + (kk & 3) * 32) >> 4), kmaj_hi, idesc_qk);
-                tc_commit_pair_elect(&ctl->k_empty[kpar]);
-                tc_commit_pair_elect(&ctl->s_full[sbuf]);
+                tc_commit_pair_elect(&ctl->k_empty[kpar], pair_mask);
+                tc_commit_pair_elect(&ctl->s_full[sbuf], pair_mask);
             };
             // O += P(t) V(t): 4 k-steps of 16 tokens, two N=256 instructions each
             auto issue_pv = [&](auto par_tag, bool first) {
@@ -524,7 +639,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
                     tc_mma_pair_elect<true>(tmem_u + kColO, ak, kmaj_hi, bk, v_hi, idesc_pv);
                     tc_mma_pair_elect<true>(tmem_u + kColO + 128, ak, kmaj_hi, bk + ((2 * kPanelBytes) >> 4), v_hi, idesc_pv);
                 }
-                tc_commit_pair_elect(&ctl->pv_done[par]);
+                tc_commit_pair_elect(&ctl->pv_done[par], pair_mask);
             };
             // Q K^T runs two tiles ahead of P V (three S buffers), so the chain S ready -> softmax ->
             // P -> P V of a tile has two tile times to complete before the tensor pipe needs it.
@@ -591,9 +706,9 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         const int half = quarter >> 1;                      // token half of S / column half of O
         const int part = half * 2 + sub;                    // which quarter of the tile's tokens
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-        const uint32_t s_empty_leader = map_to_rank(smem_u32(&ctl->s_empty[0]), 0);   // [1], [2] follow at +8, +16
-        const uint32_t p_full_leader0 = map_to_rank(smem_u32(&ctl->p_full[0]), 0);
-        const uint32_t p_full_leader1 = map_to_rank(smem_u32(&ctl->p_full[1]), 0);
+        const uint32_t s_empty_leader = map_to_rank(smem_u32(&ctl->s_empty[0]), leader);   // [1], [2] follow at +8, +16
+        const uint32_t p_full_leader0 = map_to_rank(smem_u32(&ctl->p_full[0]), leader);
+        const uint32_t p_full_leader1 = map_to_rank(smem_u32(&ctl->p_full[1]), leader);
         float m_ref = -INFINITY, l = 0.f;
         bool ok = true;
         for (int i = 0; i < tiles; ++i) {
@@ -697,6 +812,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         if (ok) {
             ok = mbar_wait(&ctl->pv_done[(tiles - 1) & 1], ((tiles - 1) >> 1) & 1);
             OMNI_STAMP(0x48, 0);
+            OMNI_SPAN(2);
             ok = __all_sync(0xffffffffu, ok);
         }
         if (ok) {
@@ -706,72 +822,95 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
             ok = mbar_wait(&ctl->x_bar, tiles & 1);
             ok = __all_sync(0xffffffffu, ok);
         }
-        if (ok) {
-            // The 64 output rows of this CTA are one contiguous block of global memory.  They are
-            // staged in shared memory (all operand buffers are dead by now; the row pitch is padded
-            // by 16 B so that the 32 rows a warp writes at once fall in different banks) and then
-            // written out with fully coalesced stores instead of scattered 16-byte ones.
+        if (ok && p.cluster_merge) {
+            // the result stays in tensor memory: the exchange after the main loop scales it and
+            // hands half of it to the CTA that serves the same heads in the other split
+            const float lt = (ctl->xchg[tiles & 1][0][row] + ctl->xchg[tiles & 1][1][row]) +
+                             (ctl->xchg[tiles & 1][2][row] + ctl->xchg[tiles & 1][3][row]);
+            cm_inv = lt > 0.f ? 1.f / lt : 0.f;
+            cm_lse = lt > 0.f ? (m_ref + log2f(lt)) * kLn2 : -INFINITY;
+        } else if (ok) {
+            // Each warp owns 32 rows x 128 value columns of the result.  It moves them out in rounds
+            // of 128 bytes per row: tensor memory -> registers (scaled) -> a warp-private staging
+            // tile in shared memory (all operand buffers are dead by now; 144-byte pitch, so neither
+            // the row-per-lane writes nor the line-per-8-lanes reads conflict) -> global memory as
+            // whole 128-byte lines, four rows per instruction.  The staging tile is double
+            // buffered and no CTA-wide barrier is needed, so the stores of one round overlap the
+            // tensor-memory reads of the next.
             tc_fence_after();
             const float lt = (ctl->xchg[tiles & 1][0][row] + ctl->xchg[tiles & 1][1][row]) +
                              (ctl->xchg[tiles & 1][2][row] + ctl->xchg[tiles & 1][3][row]);
             const float inv = lt > 0.f ? 1.f / lt : 0.f;
             const int h = h0 + row;
-            const bool store = h < p.heads;
             const bool final_out = p.splits == 1;
             const size_t u = final_out ? ((size_t)b * p.heads + h) : (((size_t)b * p.splits + s) * p.heads + h);
-            const uint32_t row_bytes = final_out ? kDv * 2 : kDv * 4, pitch = row_bytes + 16;
-            uint8_t *stage_row = smem + (size_t)row * pitch + part * (row_bytes / 4);
+            constexpr uint32_t kStagePitch = 144, kStageBytes = 32 * kStagePitch;
+            const int widx = sub * 4 + ((warp - 2) & 3);                         // 0..7
+            uint8_t *stage = smem + (size_t)widx * 2 * kStageBytes;
+            const uint32_t row_bytes = final_out ? kDv * 2 : kDv * 4;
+            const int row0 = (quarter & 1) * 32;                                  // first head row of this warp
+            // global address of (row0, this warp's first value column)
+            const size_t u0 = final_out ? ((size_t)b * p.heads + h0 + row0) : (((size_t)b * p.splits + s) * p.heads + h0 + row0);
+            uint8_t *gbase = (final_out ? reinterpret_cast<uint8_t *>(p.out + u0 * kDv)
+                                        : reinterpret_cast<uint8_t *>(p.part_out + u0 * kDv)) + part * (row_bytes / 4);
+            const int rows_here = max(0, min(32, head_rows - row0));              // rows of this warp that exist
+            const int rounds = final_out ? 2 : 4;
 #pragma unroll 1
-            for (int c = 0; c < 128; c += 32) {
-                uint32_t ov[32];
+            for (int q = 0; q < rounds; ++q) {
+                uint8_t *buf = stage + (q & 1) * kStageBytes;
+                uint4 *mine = reinterpret_cast<uint4 *>(buf + lane * kStagePitch);
                 __syncwarp();
-                tc_ld32(tmem + lane_base + kColO + 128 * sub + c, ov);
-                tc_wait_ld();
                 if (final_out) {
-                    uint4 *o = reinterpret_cast<uint4 *>(stage_row + c * 2);
+                    // 64 columns -> 128 bytes of bf16
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        uint4 w;
-                        w.x = pack_bf16(__uint_as_float(ov[8 * j]) * inv, __uint_as_float(ov[8 * j + 1]) * inv);
-                        w.y = pack_bf16(__uint_as_float(ov[8 * j + 2]) * inv, __uint_as_float(ov[8 * j + 3]) * inv);
-                        w.z = pack_bf16(__uint_as_float(ov[8 * j + 4]) * inv, __uint_as_float(ov[8 * j + 5]) * inv);
-                        w.w = pack_bf16(__uint_as_float(ov[8 * j + 6]) * inv, __uint_as_float(ov[8 * j + 7]) * inv);
-                        o[j] = w;
+                    for (int c2 = 0; c2 < 2; ++c2) {
+                        uint32_t ov[32];
+                        tc_ld32(tmem + lane_base + kColO + 128 * sub + q * 64 + c2 * 32, ov);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            uint4 w;
+                            w.x = pack_bf16(__uint_as_float(ov[8 * j]) * inv, __uint_as_float(ov[8 * j + 1]) * inv);
+                            w.y = pack_bf16(__uint_as_float(ov[8 * j + 2]) * inv, __uint_as_float(ov[8 * j + 3]) * inv);
+                            w.z = pack_bf16(__uint_as_float(ov[8 * j + 4]) * inv, __uint_as_float(ov[8 * j + 5]) * inv);
+                            w.w = pack_bf16(__uint_as_float(ov[8 * j + 6]) * inv, __uint_as_float(ov[8 * j + 7]) * inv);
+                            mine[c2 * 4 + j] = w;
+                        }
                     }
                 } else {
-                    float4 *o = reinterpret_cast<float4 *>(stage_row + c * 4);
+                    // 32 columns -> 128 bytes of fp32
+                    uint32_t ov[32];
+                    tc_ld32(tmem + lane_base + kColO + 128 * sub + q * 32, ov);
+                    tc_wait_ld();
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
-                        o[j] = make_float4(__uint_as_float(ov[4 * j]) * inv, __uint_as_float(ov[4 * j + 1]) * inv,
-                                           __uint_as_float(ov[4 * j + 2]) * inv, __uint_as_float(ov[4 * j + 3]) * inv);
+                        mine[j] = make_uint4(__float_as_uint(__uint_as_float(ov[4 * j]) * inv),
+                                             __float_as_uint(__uint_as_float(ov[4 * j + 1]) * inv),
+                                             __float_as_uint(__uint_as_float(ov[4 * j + 2]) * inv),
+                                             __float_as_uint(__uint_as_float(ov[4 * j + 3]) * inv));
+                }
+                __syncwarp();
+                uint8_t *gq = gbase + q * 128;
+                uint4 v[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    v[k] = *reinterpret_cast<const uint4 *>(buf + (4 * k + (lane >> 3)) * kStagePitch + (lane & 7) * 16);
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const int r = 4 * k + (lane >> 3);
+                    if (r < rows_here) *reinterpret_cast<uint4 *>(gq + (size_t)r * row_bytes + (lane & 7) * 16) = v[k];
                 }
             }
-            if (store && part == 0) {
+            if (h < p.heads && part == 0) {
                 const float lse = lt > 0.f ? (m_ref + log2f(lt)) * kLn2 : -INFINITY;
                 if (final_out)
                     p.lse[u] = lse;
                 else
                     p.part_lse[u] = lse;
             }
-            // all rows staged -> the 256 threads copy the block out in 16-byte pieces, consecutive
-            // threads to consecutive addresses (one bulk copy per row would cost 64 copy-engine
-            // instructions, ~3 us at the engine's instruction rate)
-            mbar_arrive(&ctl->x_bar);
-            ok = mbar_wait(&ctl->x_bar, (tiles + 1) & 1);
-            ok = __all_sync(0xffffffffu, ok);
-            if (ok) {
-                const int t = (sub * 4 + ((warp - 2) & 3)) * 32 + lane;          // 0..255
-                const size_t u0 = final_out ? ((size_t)b * p.heads + h0) : (((size_t)b * p.splits + s) * p.heads + h0);
-                uint8_t *dst = final_out ? reinterpret_cast<uint8_t *>(p.out + u0 * kDv)
-                                         : reinterpret_cast<uint8_t *>(p.part_out + u0 * kDv);
-                const uint32_t total = (uint32_t)head_rows * row_bytes;
-                for (uint32_t off = (uint32_t)t * 16; off < total; off += 256 * 16) {
-                    const uint32_t r = off / row_bytes, c = off % row_bytes;
-                    *reinterpret_cast<uint4 *>(dst + off) = *reinterpret_cast<const uint4 *>(smem + (size_t)r * pitch + c);
-                }
-                if (!final_out) __threadfence();       // partial results visible before this CTA is counted
-                OMNI_STAMP(0x49, 0);
-            }
+            // with the in-kernel merge the partial results must be visible before this CTA is counted
+            if (!final_out && p.counters != nullptr) __threadfence();
+            OMNI_STAMP(0x49, 0);
         }
         if (!ok && lane == 0) {
             flag_status(p.status, OMNI_DEV_TIMEOUT | OMNI_DEV_ROLE_SOFTMAX);
@@ -784,15 +923,21 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         // a wait ran out: give copies that are still in flight time to land before anyone exits
         for (int i = 0; i < 200; ++i) __nanosleep(1000);
     }
+    if (p.cluster_merge) cluster_merge_exchange(p, ctl, smem, tmem, b, s, crank, h0, head_rows, active, cm_lse, cm_inv);
     tc_fence_before();
     __syncthreads();
+    if (!active) {
+        // no tensor memory to give back; leave together with the rest of the cluster
+        cluster_sync_all();
+        return;
+    }
     // Tensor memory was allocated for the pair, so it is released only when both CTAs are done
     // with it.  The rendezvous is an mbarrier in each CTA that both CTAs arrive on (the hardware
     // cluster barrier took 6-9 us at this point); warp 1 stays until the peer's arrival has
     // landed, which also keeps this CTA's shared memory alive for it.
     if (threadIdx.x == 0) {
         mbar_arrive(&ctl->exit_bar);
-        mbar_arrive_cluster(map_to_rank(smem_u32(&ctl->exit_bar), rank ^ 1));
+        mbar_arrive_cluster(map_to_rank(smem_u32(&ctl->exit_bar), peer));
     }
     if (warp == 1) {
         mbar_wait(&ctl->exit_bar, 0);
@@ -800,11 +945,47 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
+    // the bulk copy a CTA sent to its partner reads this CTA's shared memory: nobody leaves
+    // before every CTA of the cluster has received its block
+    if (p.cluster_merge) cluster_sync_all();
     // ---- split merge by whichever CTA finishes a (request, head half) last ---------------
     OMNI_STAMP(0x02, 0);
     if (p.splits > 1 && p.counters != nullptr)
         merge_if_last(p, b, (int)rank, 2, h0, head_rows, reinterpret_cast<float *>(smem), &ctl->merge_flag);
     OMNI_STAMP(0x03, 0);
+    OMNI_SPAN(3);
+}
+
+// Clusters of two pairs (cluster merge) that can be resident at once on the current device, or 0.
+inline int tc2_max_merge_clusters()
+{
+    static int cached[64];
+    static bool known[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    if (!known[dev]) {
+        int n = 0;
+        if (cudaFuncSetAttribute(tc2_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kC2SmemBytes) == cudaSuccess) {
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(4 * 64);
+            cfg.blockDim = dim3(kC2Threads);
+            cfg.dynamicSmemBytes = kC2SmemBytes;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = 4;
+            attr[0].val.clusterDim.y = 1;
+            attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            if (cudaOccupancyMaxActiveClusters(&n, tc2_decode_kernel, &cfg) != cudaSuccess) {
+                cudaGetLastError();
+                n = 0;
+            }
+        }
+        cached[dev] = n;
+        known[dev] = true;
+    }
+    return cached[dev];
 }
 
 inline omni_status_t launch_tc2_decode(const DecodeParams &p, cudaStream_t stream)
@@ -829,13 +1010,17 @@ inline omni_status_t launch_tc2_decode(const DecodeParams &p, cudaStream_t strea
     cfg.blockDim = dim3(kC2Threads);
     cfg.dynamicSmemBytes = kC2SmemBytes;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.x = p.cluster_merge ? 4 : 2;      // cluster merge: both splits of a request in one cluster
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    // the launch may overlap the tail of the previous kernel in the stream (the kernel waits
+    // before its first global access), which hides the launch latency between decode steps
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, tc2_decode_kernel, q_map, kv_map, kv_k_map, kv_v_map, kv_tile_map, p) == cudaSuccess
                ? OMNI_OK
                : OMNI_ERR_CUDA;

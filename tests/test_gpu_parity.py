@@ -13,7 +13,8 @@ from parity import check_workload, compare, oracle_subset, run_gpu
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
-IMPLS = {"simt": B.OMNI_FLAG_SIMT, "tc": 0, "tc_fused_merge": B.OMNI_FLAG_FUSED_MERGE}
+IMPLS = {"simt": B.OMNI_FLAG_SIMT, "tc": 0, "tc_fused_merge": B.OMNI_FLAG_FUSED_MERGE,
+         "tc_no_cluster_merge": B.OMNI_FLAG_NO_CLUSTER_MERGE}
 
 
 @pytest.fixture(params=list(IMPLS))
@@ -47,7 +48,7 @@ def test_ragged_lengths_and_tails(flags):
     lens = [0, 1, 2, 63, 64, 65, 127, 129, 300, 513]
     sels = [rng.permutation(16 * 64)[:n] for n in lens]
     w = _custom("ragged_tails", 41, 128, [16] * len(lens), sels)
-    for s in (0, 1, 4):
+    for s in (0, 1, 2, 4):
         stats, plan = check_workload(w, flags, num_splits=s, what="ragged tails S=%d" % s)
         assert torch.all(plan.out[0] == 0) and torch.all(torch.isneginf(plan.lse[0]))
 
@@ -149,7 +150,7 @@ def test_rows_outside_the_selection_are_never_used(flags):
     keep = torch.zeros(w.num_pages * 64, dtype=torch.bool, device=DEV)
     keep[torch.from_numpy(rows[rows >= 0]).to(DEV)] = True
     w.kv_cache.view(-1, 576)[~keep] = float("nan")
-    for s in (0, 1, 3):
+    for s in (0, 1, 2, 3):
         check_workload(w, flags, num_splits=s, what="nan outside S=%d" % s)
 
 
