@@ -87,6 +87,15 @@ const char *omni_status_string(omni_status_t status);
 int32_t omni_sparse_mla_num_splits(const omni_mla_desc_t *desc);
 
 /*
+ * Kernels one omni_sparse_mla_decode call launches for this descriptor on the current device:
+ * the decode kernel, plus the split-KV merge kernel unless the splits are merged inside the
+ * decode kernel (two splits per request whose CTA clusters are all resident at once, or
+ * OMNI_FLAG_FUSED_MERGE), plus the validation kernel if OMNI_FLAG_VALIDATE is set.  Returns 0
+ * on a bad descriptor.
+ */
+int32_t omni_sparse_mla_num_launches(const omni_mla_desc_t *desc);
+
+/*
  * Bytes of device workspace omni_sparse_mla_decode needs for this descriptor: room for the
  * fp32 partial outputs and partial log-sum-exps of every (request, split) and for the
  * arrival counters of the in-kernel merge.  Returns 0 on a bad descriptor.  The workspace

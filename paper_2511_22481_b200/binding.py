@@ -25,7 +25,7 @@ OMNI_FLAG_FUSED_MERGE = 4
 OMNI_FLAG_NO_CLUSTER_MERGE = 8
 
 EXPORTS = (
-    "omni_version", "omni_status_string", "omni_sparse_mla_num_splits",
+    "omni_version", "omni_status_string", "omni_sparse_mla_num_splits", "omni_sparse_mla_num_launches",
     "omni_sparse_mla_workspace_bytes", "omni_sparse_mla_decode", "omni_sparse_mla_combine",
     "omni_sparse_mla_validate", "omni_sparse_mla_resolve_rows",
     "omni_sparse_mla_host_staging_bytes", "omni_sparse_mla_decode_host",
@@ -75,6 +75,8 @@ def load() -> ctypes.CDLL:
     lib.omni_status_string.argtypes = [ctypes.c_int]
     lib.omni_sparse_mla_num_splits.restype = i32
     lib.omni_sparse_mla_num_splits.argtypes = [dp]
+    lib.omni_sparse_mla_num_launches.restype = i32
+    lib.omni_sparse_mla_num_launches.argtypes = [dp]
     lib.omni_sparse_mla_workspace_bytes.restype = sz
     lib.omni_sparse_mla_workspace_bytes.argtypes = [dp]
     lib.omni_sparse_mla_decode.restype = ctypes.c_int
@@ -137,6 +139,10 @@ def _check(code, where):
 
 def omni_sparse_mla_num_splits(desc: OmniDesc) -> int:
     return int(load().omni_sparse_mla_num_splits(ctypes.byref(desc)))
+
+
+def omni_sparse_mla_num_launches(desc: OmniDesc) -> int:
+    return int(load().omni_sparse_mla_num_launches(ctypes.byref(desc)))
 
 
 def omni_sparse_mla_workspace_bytes(desc: OmniDesc) -> int:

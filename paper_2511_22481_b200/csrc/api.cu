@@ -94,6 +94,14 @@ int choose_splits(const omni_mla_desc_t *d, int sm_count)
     return best;
 }
 
+// Two splits of a request can be merged inside a cluster of two CTA pairs as long as all those
+// clusters are resident at once.
+bool merge_in_cluster(const omni_mla_desc_t *d, int splits)
+{
+    return splits == 2 && use_pair_kernel(d) && !(d->flags & (OMNI_FLAG_FUSED_MERGE | OMNI_FLAG_NO_CLUSTER_MERGE)) &&
+           d->batch <= tc2_max_merge_clusters();
+}
+
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 size_t part_out_bytes(const omni_mla_desc_t *d, int splits)
@@ -202,6 +210,15 @@ int32_t omni_sparse_mla_num_splits(const omni_mla_desc_t *desc)
     return choose_splits(desc, device_info().sm_count);
 }
 
+int32_t omni_sparse_mla_num_launches(const omni_mla_desc_t *desc)
+{
+    if (!desc_ok(desc)) return 0;
+    const int s = choose_splits(desc, device_info().sm_count);
+    int n = 1 + ((desc->flags & OMNI_FLAG_VALIDATE) ? 1 : 0);
+    if (s > 1 && !merge_in_cluster(desc, s) && !(use_pair_kernel(desc) && (desc->flags & OMNI_FLAG_FUSED_MERGE))) ++n;
+    return n;
+}
+
 size_t omni_sparse_mla_workspace_bytes(const omni_mla_desc_t *desc)
 {
     if (!desc_ok(desc)) return 0;
@@ -253,9 +270,7 @@ omni_status_t omni_sparse_mla_decode(const omni_mla_desc_t *desc, const void *q,
     p.cluster_merge = 0;
     // Two splits of a request can be merged inside a cluster of two CTA pairs, without partial
     // results in global memory, as long as all those clusters are resident at once.
-    if (splits == 2 && use_pair_kernel(desc) && !(desc->flags & (OMNI_FLAG_FUSED_MERGE | OMNI_FLAG_NO_CLUSTER_MERGE)) &&
-        desc->batch <= tc2_max_merge_clusters())
-        p.cluster_merge = 1;
+    if (merge_in_cluster(desc, splits)) p.cluster_merge = 1;
     if (splits > 1 && merge_in_kernel(desc)) {
         p.counters = reinterpret_cast<int32_t *>(static_cast<char *>(workspace) + part_out_bytes(desc, splits) +
                                                  part_lse_bytes(desc, splits));
