@@ -83,6 +83,7 @@ struct C2Control {
     uint32_t merge_flag;
     int32_t k_progress;                  // tiles whose K loads the producer has started (L2 prefetch pacing)
     uint64_t recv_bar;                   // cluster merge: the partner's block has arrived
+    uint64_t ready_bar;                  // cluster merge: the partner's main loop is over
     float xlse[2][64];                   // cluster merge: log-sum-exp of either split, per head row
 };
 static_assert(sizeof(C2Control) <= kC2SmemCtlBytes, "control block too large");
@@ -179,45 +180,35 @@ __device__ __forceinline__ void tc_commit_pair_elect(uint64_t *bar, uint16_t bot
 // merge).  CTA `crank` and its partner `crank ^ 2` serve the same 64 heads in the two splits.
 // Instead of writing fp32 partial results to global memory for a second kernel to read back,
 // the two exchange what the other needs through distributed shared memory:
-//   1. each tells the other the log-sum-exp of its split for every head row;
-//   2. each scales its accumulator by exp(lse_own - lse_total) / row sum, keeps the 256 value
-//      columns it will finish (split 0: columns 0..255, split 1: 256..511) and sends the other
-//      256 to the partner with one bulk shared-memory-to-shared-memory copy;
-//   3. each adds what it received to what it kept and stores its half of the final rows.
-// Called by every thread of every CTA of the cluster after the main loop; all operand buffers
-// are dead by then (the cluster barrier in step 1 is what tells a CTA that this also holds for
-// its partner, whose shared memory it writes to).
+//   1. each normalises its accumulator by its row sums, keeps the 256 value columns it will
+//      finish (split 0: columns 0..255, split 1: 256..511) and sends the other 256, followed by
+//      the log-sum-exp of its split for every head row, to the partner with one bulk
+//      shared-memory-to-shared-memory copy;
+//   2. each weighs what it kept and what it received by exp(lse_split - lse_total), adds them
+//      and stores its half of the final rows.
+// The copy lands in shared memory that held the partner's operand tiles, so it is not sent
+// before the partner has said that its main loop is over (`ready_bar`, a remote arrive that the
+// partner fires as soon as its last P V has retired, while this CTA is still staging).
+// Called by every thread of the CTA after the main loop.
 __device__ __forceinline__ void cluster_merge_exchange(const DecodeParams &p, C2Control *ctl, uint8_t *smem,
                                                        uint32_t tmem, int b, int s, uint32_t crank, int h0,
                                                        int head_rows, bool active, float cm_lse, float cm_inv)
 {
     constexpr uint32_t kSliceBytes = 256 * 4;            // half of a row's value columns, fp32
     constexpr uint32_t kPitch = kSliceBytes + 16;        // row-per-lane 16-byte accesses do not conflict
-    constexpr uint32_t kBlockBytes = 64 * kPitch;        // 66,560
+    constexpr uint32_t kRowsBytes = 64 * kPitch;         // 66,560
+    constexpr uint32_t kBlockBytes = kRowsBytes + 256;   // + 64 log-sum-exps
     static_assert(3 * kBlockBytes <= kC2SmemCtl, "exchange tiles must fit below the control block");
     uint8_t *send = smem, *keep = smem + kBlockBytes, *recv = smem + 2 * kBlockBytes;
     const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;
     const bool is_softmax = (warp >= 2 && warp <= 5) || warp >= 8;
+    if (!is_softmax) return;
     const int quarter = warp & 3, sub = warp >= 8 ? 1 : 0;
     const int row = (quarter & 1) * 32 + lane, part = (quarter >> 1) * 2 + sub;
     const uint32_t partner = crank ^ 2u;
+    // an empty split never ran a main loop: its shared memory is free from the start
+    if (!active && warp == 2 && lane == 0) mbar_arrive_cluster(map_to_rank(smem_u32(&ctl->ready_bar), partner));
 
-    if (is_softmax && part == 0) {
-        ctl->xlse[s][row] = cm_lse;
-        const uint32_t remote = map_to_rank(smem_u32(&ctl->xlse[s][row]), partner);
-        asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(cm_lse) : "memory");
-    }
-    cluster_sync_all();
-    if (!is_softmax) return;
-
-    const float a0 = ctl->xlse[0][row], a1 = ctl->xlse[1][row];
-    const float mx = fmaxf(a0, a1);
-    float total = -INFINITY, w = 0.f;
-    if (mx > -INFINITY) {
-        total = mx + logf(exp2f((a0 - mx) * kLog2e) + exp2f((a1 - mx) * kLog2e));
-        if (cm_lse > -INFINITY) w = exp2f((cm_lse - total) * kLog2e);
-    }
-    const float f = w * cm_inv;
     // this thread's 128 value columns are finished by split `part / 2`
     uint8_t *tile = ((part >> 1) == s ? keep : send) + (size_t)row * kPitch + (part & 1) * 512;
     const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
@@ -232,45 +223,72 @@ __device__ __forceinline__ void cluster_merge_exchange(const DecodeParams &p, C2
         uint4 *o = reinterpret_cast<uint4 *>(tile + q * 128);
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-            // a weight of zero (empty or fully masked split) contributes exact zeros
-            o[j] = (active && f != 0.f)
-                       ? make_uint4(__float_as_uint(__uint_as_float(ov[4 * j]) * f), __float_as_uint(__uint_as_float(ov[4 * j + 1]) * f),
-                                    __float_as_uint(__uint_as_float(ov[4 * j + 2]) * f), __float_as_uint(__uint_as_float(ov[4 * j + 3]) * f))
+            // an empty or fully masked split contributes exact zeros
+            o[j] = (active && cm_inv != 0.f)
+                       ? make_uint4(__float_as_uint(__uint_as_float(ov[4 * j]) * cm_inv),
+                                    __float_as_uint(__uint_as_float(ov[4 * j + 1]) * cm_inv),
+                                    __float_as_uint(__uint_as_float(ov[4 * j + 2]) * cm_inv),
+                                    __float_as_uint(__uint_as_float(ov[4 * j + 3]) * cm_inv))
                        : make_uint4(0u, 0u, 0u, 0u);
         }
     }
+    if (part == 0) reinterpret_cast<float *>(send + kRowsBytes)[row] = cm_lse;
     tc_fence_before();
     fence_async_smem();                                   // the bulk copy reads what the threads wrote
     asm volatile("bar.sync 1, 256;" ::: "memory");         // the eight softmax warps
-    if (warp == 2 && lane == 0) {
-        mbar_expect_tx(&ctl->recv_bar, kBlockBytes);
-        const uint32_t dst = map_to_rank(smem_u32(recv), partner);
-        const uint32_t bar = map_to_rank(smem_u32(&ctl->recv_bar), partner);
-        asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                     ::"r"(dst), "r"(smem_u32(send)), "r"(kBlockBytes), "r"(bar)
-                     : "memory");
+    bool ok = true;
+    if (warp == 2) {
+        ok = mbar_wait(&ctl->ready_bar, 0);               // the partner's operand tiles are dead
+        ok = __all_sync(0xffffffffu, ok);
+        if (ok && lane == 0) {
+            mbar_expect_tx(&ctl->recv_bar, kBlockBytes);
+            const uint32_t dst = map_to_rank(smem_u32(recv), partner);
+            const uint32_t bar = map_to_rank(smem_u32(&ctl->recv_bar), partner);
+            asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(dst), "r"(smem_u32(send)), "r"(kBlockBytes), "r"(bar)
+                         : "memory");
+        }
     }
-    bool ok = mbar_wait(&ctl->recv_bar, 0);
+    ok = ok && mbar_wait(&ctl->recv_bar, 0);
     ok = __all_sync(0xffffffffu, ok);
     if (!ok) {
         if (lane == 0) flag_status(p.status, OMNI_DEV_TIMEOUT | OMNI_DEV_ROLE_SOFTMAX);
         return;
     }
+    // weights of the two splits per head row (in place of the log-sum-exps), final log-sum-exp
+    if (part == 0) {
+        const float other = reinterpret_cast<const float *>(recv + kRowsBytes)[row];
+        const float mx = fmaxf(cm_lse, other);
+        float total = -INFINITY, w_own = 0.f, w_other = 0.f;
+        if (mx > -INFINITY) {
+            total = mx + logf(exp2f((cm_lse - mx) * kLog2e) + exp2f((other - mx) * kLog2e));
+            if (cm_lse > -INFINITY) w_own = exp2f((cm_lse - total) * kLog2e);
+            if (other > -INFINITY) w_other = exp2f((other - total) * kLog2e);
+        }
+        ctl->xlse[0][row] = w_own;
+        ctl->xlse[1][row] = w_other;
+        if (s == 0 && row < head_rows) p.lse[(size_t)b * p.heads + h0 + row] = total;
+    }
+    asm volatile("bar.sync 1, 256;" ::: "memory");
     // kept + received -> bf16, 16 output bytes (8 columns) per item, consecutive threads along a row
     const int t = (sub * 4 + ((warp - 2) & 3)) * 32 + lane;          // 0..255
     for (int item = t; item < head_rows * 32; item += 256) {
         const int r = item >> 5, c = item & 31;
+        const float wk = ctl->xlse[0][r], wr = ctl->xlse[1][r];
         const uint4 *k4 = reinterpret_cast<const uint4 *>(keep + (size_t)r * kPitch + c * 32);
         const uint4 *r4 = reinterpret_cast<const uint4 *>(recv + (size_t)r * kPitch + c * 32);
         const uint4 k0 = k4[0], k1 = k4[1], r0 = r4[0], r1 = r4[1];
+        // a weight of zero must not meet a non-finite partner value
+        auto mix = [&](uint32_t kv, uint32_t rv) {
+            return (wk != 0.f ? wk * __uint_as_float(kv) : 0.f) + (wr != 0.f ? wr * __uint_as_float(rv) : 0.f);
+        };
         uint4 o;
-        o.x = pack_bf16(__uint_as_float(k0.x) + __uint_as_float(r0.x), __uint_as_float(k0.y) + __uint_as_float(r0.y));
-        o.y = pack_bf16(__uint_as_float(k0.z) + __uint_as_float(r0.z), __uint_as_float(k0.w) + __uint_as_float(r0.w));
-        o.z = pack_bf16(__uint_as_float(k1.x) + __uint_as_float(r1.x), __uint_as_float(k1.y) + __uint_as_float(r1.y));
-        o.w = pack_bf16(__uint_as_float(k1.z) + __uint_as_float(r1.z), __uint_as_float(k1.w) + __uint_as_float(r1.w));
+        o.x = pack_bf16(mix(k0.x, r0.x), mix(k0.y, r0.y));
+        o.y = pack_bf16(mix(k0.z, r0.z), mix(k0.w, r0.w));
+        o.z = pack_bf16(mix(k1.x, r1.x), mix(k1.y, r1.y));
+        o.w = pack_bf16(mix(k1.z, r1.z), mix(k1.w, r1.w));
         *reinterpret_cast<uint4 *>(p.out + ((size_t)b * p.heads + h0 + r) * kDv + s * 256 + c * 8) = o;
     }
-    if (s == 0 && part == 0 && row < head_rows) p.lse[(size_t)b * p.heads + h0 + row] = total;
 }
 
 __global__ void __launch_bounds__(kC2Threads, 1)
@@ -360,6 +378,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         mbar_init(&ctl->x_bar, 256);
         mbar_init(&ctl->exit_bar, 2);
         mbar_init(&ctl->recv_bar, 1);
+        mbar_init(&ctl->ready_bar, 1);
         ctl->abort = 0;
         ctl->k_progress = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -823,7 +842,10 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
             ok = __all_sync(0xffffffffu, ok);
         }
         if (ok && p.cluster_merge) {
-            // the result stays in tensor memory: the exchange after the main loop scales it and
+            // every MMA of the pair has retired and every copy has landed: the partner in the other
+            // split may overwrite this CTA's operand tiles from now on
+            if (warp == 2 && lane == 0) mbar_arrive_cluster(map_to_rank(smem_u32(&ctl->ready_bar), crank ^ 2u));
+            // the result stays in tensor memory: the exchange after the main loop normalises it and
             // hands half of it to the CTA that serves the same heads in the other split
             const float lt = (ctl->xchg[tiles & 1][0][row] + ctl->xchg[tiles & 1][1][row]) +
                              (ctl->xchg[tiles & 1][2][row] + ctl->xchg[tiles & 1][3][row]);
@@ -928,7 +950,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     __syncthreads();
     if (!active) {
         // no tensor memory to give back; leave together with the rest of the cluster
-        cluster_sync_all();
+        cluster_sync_relaxed();
         return;
     }
     // Tensor memory was allocated for the pair, so it is released only when both CTAs are done
@@ -947,7 +969,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     }
     // the bulk copy a CTA sent to its partner reads this CTA's shared memory: nobody leaves
     // before every CTA of the cluster has received its block
-    if (p.cluster_merge) cluster_sync_all();
+    if (p.cluster_merge) cluster_sync_relaxed();
     // ---- split merge by whichever CTA finishes a (request, head half) last ---------------
     OMNI_STAMP(0x02, 0);
     if (p.splits > 1 && p.counters != nullptr)
