@@ -68,10 +68,21 @@ int units_per_request(const omni_mla_desc_t *d)
     return (d->num_heads + kTcHeads - 1) / kTcHeads;
 }
 
+// Two splits of a request can be merged inside a cluster of two CTA pairs as long as all those
+// clusters are resident at once.
+bool merge_in_cluster(const omni_mla_desc_t *d, int splits)
+{
+    return splits == 2 && use_pair_kernel(d) && !(d->flags & (OMNI_FLAG_FUSED_MERGE | OMNI_FLAG_NO_CLUSTER_MERGE)) &&
+           d->batch <= tc2_max_merge_clusters();
+}
+
 // Pick the number of split-KV partitions per request.  The kernel's work units run in waves over
-// the SMs; a unit costs a fixed part (set-up, first-tile latency, epilogue: about 6 tile times as
-// measured) plus one tile time per 64-token granule, and splitting at all costs about 6 more tile
-// times (partials written and merged).  Minimise waves * (granules per unit + 6) + merge.
+// the SMs.  In units of one tile time (64 tokens), as measured: a unit costs a fixed part of about
+// 6 (set-up, first-tile latency, epilogue) plus one per granule; a unit that writes fp32 partial
+// results to global memory for a later merge costs about 6 more (256 KiB written and read back
+// against 72 KiB per tile), and so does the merge kernel at the end.  Two splits merged inside a
+// cluster of two CTA pairs avoid the partial results and pay about 5 for the exchange.
+// Minimise waves * (granules per unit + fixed parts) + merge.
 int choose_splits(const omni_mla_desc_t *d, int sm_count)
 {
     if (d->num_splits >= 1) return d->num_splits;
@@ -85,21 +96,19 @@ int choose_splits(const omni_mla_desc_t *d, int sm_count)
     for (int s = 1; s <= kMaxSplits && s <= granules; ++s) {
         const long waves = (units * s + sm_count - 1) / sm_count;
         const long per = (granules + s - 1) / s;
-        const long cost = waves * (per + 6) + (s > 1 ? 6 : 0);
+        long cost;
+        if (s == 1)
+            cost = waves * (per + 6);
+        else if (merge_in_cluster(d, s))
+            cost = waves * (per + 6) + 5;
+        else
+            cost = waves * (per + 12) + 6;
         if (best_cost < 0 || cost < best_cost) {
             best_cost = cost;
             best = s;
         }
     }
     return best;
-}
-
-// Two splits of a request can be merged inside a cluster of two CTA pairs as long as all those
-// clusters are resident at once.
-bool merge_in_cluster(const omni_mla_desc_t *d, int splits)
-{
-    return splits == 2 && use_pair_kernel(d) && !(d->flags & (OMNI_FLAG_FUSED_MERGE | OMNI_FLAG_NO_CLUSTER_MERGE)) &&
-           d->batch <= tc2_max_merge_clusters();
 }
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }

@@ -300,6 +300,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     uint8_t *smem = smem_raw;
     if (smem_u32(smem_raw) & 1023u) {
         // the swizzled operand layouts need a 1024-byte aligned base; never seen otherwise, but say so
+        asm volatile("griddepcontrol.wait;" ::: "memory");
         if (threadIdx.x == 0) flag_status(p.status, OMNI_DEV_TIMEOUT);
         return;
     }
@@ -321,47 +322,8 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     OMNI_STAMP(0x04, 0);
     OMNI_SPAN(0);
 
-    // Programmatic dependent launch, both ways.  This grid may have been scheduled while the
-    // kernel before it in the stream was still finishing: nothing in global memory is touched
-    // until that kernel has completed and its writes are visible.  And the kernel after this one
-    // may be scheduled as soon as resources allow; it waits in the same way before it reads.
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    int n = __ldg(p.sel_len + b);
-    bool bad_len = false;
-    if (n < 0 || n > p.max_sel) {
-        bad_len = true;
-        n = 0;
-    }
-    int begin, end;
-    split_range(n, p.splits, s, begin, end, kC2Tile);
-    const int tiles = (end - begin + kC2Tile - 1) / kC2Tile;
-
-    const bool active = tiles > 0;
-    if (!active && bad_len && threadIdx.x == 0 && crank == 0) flag_status(p.status, OMNI_DEV_BAD_INDEX);
-    if (!active && !p.cluster_merge) {
-        // empty split (the same decision in both CTAs of the pair): zeros and -inf, no cluster work
-        for (int r = warp; r < head_rows; r += kC2Threads / 32) {
-            const int h = h0 + r;
-            if (p.splits == 1) {
-                uint4 *o = reinterpret_cast<uint4 *>(p.out + ((size_t)b * p.heads + h) * kDv);
-                for (int i = lane; i < kDv * 2 / 16; i += 32) o[i] = make_uint4(0, 0, 0, 0);
-                if (lane == 0) p.lse[(size_t)b * p.heads + h] = -INFINITY;
-            } else {
-                const size_t u = ((size_t)b * p.splits + s) * p.heads + h;
-                float4 *o = reinterpret_cast<float4 *>(p.part_out + u * kDv);
-                for (int i = lane; i < kDv / 4; i += 32) o[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (lane == 0) p.part_lse[u] = -INFINITY;
-            }
-        }
-        if (p.splits > 1 && p.counters != nullptr) {
-            __threadfence();
-            merge_if_last(p, b, (int)rank, 2, h0, head_rows, reinterpret_cast<float *>(smem), &ctl->merge_flag);
-        }
-        return;
-    }
-
-    // ---- set-up ---------------------------------------------------------------------------
+    // ---- set-up: barriers and tensor memory (nothing here touches global memory, so with a
+    // programmatic dependent launch it overlaps the tail of the kernel before this one) --------
     if (threadIdx.x == 0) {
         mbar_init(&ctl->q_full, 1);
         for (int i = 0; i < 2; ++i) {
@@ -383,7 +345,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         ctl->k_progress = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1 && active) {
+    if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)),
                      "r"(kTmemCols)
                      : "memory");
@@ -393,6 +355,42 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     __syncthreads();
     cluster_sync_all();
     tc_fence_after();
+    // Programmatic dependent launch, both ways.  This grid may have been scheduled while the
+    // kernel before it in the stream was still finishing: nothing in global memory is touched
+    // until that kernel has completed and its writes are visible.  And the kernel after this one
+    // may be scheduled as soon as resources allow; it waits in the same way before it reads.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    int n = __ldg(p.sel_len + b);
+    bool bad_len = false;
+    if (n < 0 || n > p.max_sel) {
+        bad_len = true;
+        n = 0;
+    }
+    int begin, end;
+    split_range(n, p.splits, s, begin, end, kC2Tile);
+    const int tiles = (end - begin + kC2Tile - 1) / kC2Tile;
+
+    const bool active = tiles > 0;
+    if (!active && bad_len && threadIdx.x == 0 && crank == 0) flag_status(p.status, OMNI_DEV_BAD_INDEX);
+    if (!active && !p.cluster_merge) {
+        // empty split (the same decision in both CTAs of the pair): zeros and -inf, no pipeline
+        for (int r = warp; r < head_rows; r += kC2Threads / 32) {
+            const int h = h0 + r;
+            if (p.splits == 1) {
+                uint4 *o = reinterpret_cast<uint4 *>(p.out + ((size_t)b * p.heads + h) * kDv);
+                for (int i = lane; i < kDv * 2 / 16; i += 32) o[i] = make_uint4(0, 0, 0, 0);
+                if (lane == 0) p.lse[(size_t)b * p.heads + h] = -INFINITY;
+            } else {
+                const size_t u = ((size_t)b * p.splits + s) * p.heads + h;
+                float4 *o = reinterpret_cast<float4 *>(p.part_out + u * kDv);
+                for (int i = lane; i < kDv / 4; i += 32) o[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (lane == 0) p.part_lse[u] = -INFINITY;
+            }
+        }
+        if (p.splits > 1 && p.counters != nullptr) __threadfence();
+    }
+
     const uint32_t tmem = ctl->tmem_base;
     volatile uint32_t *abort_flag = &ctl->abort;
     OMNI_STAMP(0x01, 0);
@@ -948,11 +946,6 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     if (p.cluster_merge) cluster_merge_exchange(p, ctl, smem, tmem, b, s, crank, h0, head_rows, active, cm_lse, cm_inv);
     tc_fence_before();
     __syncthreads();
-    if (!active) {
-        // no tensor memory to give back; leave together with the rest of the cluster
-        cluster_sync_relaxed();
-        return;
-    }
     // Tensor memory was allocated for the pair, so it is released only when both CTAs are done
     // with it.  The rendezvous is an mbarrier in each CTA that both CTAs arrive on (the hardware
     // cluster barrier took 6-9 us at this point); warp 1 stays until the peer's arrival has
