@@ -79,8 +79,9 @@ bool merge_in_cluster(const omni_mla_desc_t *d, int splits)
 // Pick the number of split-KV partitions per request.  The kernel's work units run in waves over
 // the SMs.  In units of one tile time (64 tokens), as measured: a unit costs a fixed part of about
 // 6 (set-up, first-tile latency, epilogue) plus one per granule; a unit that writes fp32 partial
-// results to global memory for a later merge costs about 6 more (256 KiB written and read back
-// against 72 KiB per tile), and so does the merge kernel at the end.  Two splits merged inside a
+// results to global memory for a later merge costs about 6 more when the grid runs in several
+// waves (256 KiB written and read back against 72 KiB per tile; about 2 within one wave, where
+// they stay in L2), and so does the merge kernel at the end.  Two splits merged inside a
 // cluster of two CTA pairs avoid the partial results and pay about 5 for the exchange.
 // Minimise waves * (granules per unit + fixed parts) + merge.
 int choose_splits(const omni_mla_desc_t *d, int sm_count)
@@ -102,7 +103,7 @@ int choose_splits(const omni_mla_desc_t *d, int sm_count)
         else if (merge_in_cluster(d, s))
             cost = waves * (per + 6) + 5;
         else
-            cost = waves * (per + 12) + 6;
+            cost = waves * (per + 6 + (waves > 1 ? 6 : 2)) + 6;     // partial results stay in L2 within one wave
         if (best_cost < 0 || cost < best_cost) {
             best_cost = cost;
             best = s;
