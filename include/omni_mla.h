@@ -217,8 +217,8 @@ omni_status_t omni_sparse_mla_decode_host(const omni_mla_desc_t *desc, const voi
  *     with that device current) and caches it; make that first call during start-up, before
  *     any stream capture begins;
  *   - all calls on one device share the one array, which keeps whatever the previous call left
- *     in it.  Nothing in it needs clearing (each call overwrites every partial result it
- *     reads back), but two calls that overlap on the GPU, e.g. on different streams, race on
+ *     in it.  The caller clears nothing (each call overwrites every partial result it reads
+ *     back and clears the few counters it needs at zero itself), but two calls that overlap on the GPU, e.g. on different streams, race on
  *     it: serialise them, or give the concurrent ones omni_sparse_mla_decode with separate
  *     workspaces.
  * All other arguments, results, alignment rules and status codes are those of

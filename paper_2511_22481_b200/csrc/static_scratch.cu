@@ -52,8 +52,10 @@ extern "C" omni_status_t omni_sparse_mla_decode_static(const omni_mla_desc_t *de
     if (need > (size_t)OMNI_STATIC_SCRATCH_BYTES) return OMNI_ERR_WORKSPACE;
     void *scratch = nullptr;
     if (scratch_address(&scratch) != cudaSuccess) return OMNI_ERR_CUDA;
-    // Nothing in the scratch has to start at zero: the decode kernel writes the partial result
-    // of every (request, split, head) it later merges, empty splits included.
+    // The caller has nothing to clear: the decode kernel writes the partial result of every
+    // (request, split, head) it later merges, empty splits included, and the arrival counters
+    // of the fused merge (OMNI_FLAG_FUSED_MERGE), the only words that must start at zero, are
+    // cleared on the stream by omni_sparse_mla_decode itself.
     return omni_sparse_mla_decode(desc, q, kv_cache, page_table, sel_idx, sel_len, out, lse, scratch,
                                   (size_t)OMNI_STATIC_SCRATCH_BYTES, device_status, stream);
 }
