@@ -137,6 +137,31 @@ omni_status_t omni_sparse_mla_decode(const omni_mla_desc_t *desc, const void *q,
                                      int32_t *device_status, void *stream);
 
 /*
+ * The same operation with the index set of Eq. 2 of the paper (attention sink + recent
+ * tokens) given as its two parameters instead of an index list, so that no sel_idx array
+ * has to be built or read.  Counting positions from 0, request b with context length
+ * M = ctx_len[b] attends to [0, min(N_sink, M)) united with [max(M - N_recent, 0), M); where
+ * the two ranges overlap the union is taken without repeats, so the selection is the whole
+ * context once N_sink + N_recent >= M.  The result is that of omni_sparse_mla_decode on the
+ * increasing list of those positions, bit for bit.
+ *
+ *   ctx_len    int32 [B], each in [0, max_pages_per_req * 64]; a value outside is treated like a
+ *              bad sel_len (out = 0, lse = -inf, OMNI_DEV_BAD_INDEX)
+ *   n_sink, n_recent   N_sink and N_recent of Eq. 2, >= 0
+ *   desc->max_sel      upper bound of the selection size the split-KV plan is made for; must be
+ *              at least min(n_sink + n_recent, max_pages_per_req * 64), else OMNI_ERR_SHAPE.
+ *              Workspace and split queries apply to this descriptor unchanged.
+ * OMNI_FLAG_VALIDATE is ignored (there is no index list to check; page ids are still checked
+ * where they are used).  All other arguments are those of omni_sparse_mla_decode.
+ */
+omni_status_t omni_sparse_mla_decode_sink_recent(const omni_mla_desc_t *desc, const void *q,
+                                                 const void *kv_cache, const int32_t *page_table,
+                                                 const int32_t *ctx_len, int32_t n_sink,
+                                                 int32_t n_recent, void *out, float *lse,
+                                                 void *workspace, size_t workspace_bytes,
+                                                 int32_t *device_status, void *stream);
+
+/*
  * Merge of split-KV partial results (the step that follows a partition of M into disjoint
  * ranges; Eq. 1 is recovered exactly because softmax normalisers add):
  *     lse[b,h]   = ln sum_s exp(part_lse[b,s,h])

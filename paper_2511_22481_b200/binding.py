@@ -26,7 +26,8 @@ OMNI_FLAG_NO_CLUSTER_MERGE = 8
 
 EXPORTS = (
     "omni_version", "omni_status_string", "omni_sparse_mla_num_splits", "omni_sparse_mla_num_launches",
-    "omni_sparse_mla_workspace_bytes", "omni_sparse_mla_decode", "omni_sparse_mla_combine",
+    "omni_sparse_mla_workspace_bytes", "omni_sparse_mla_decode", "omni_sparse_mla_decode_sink_recent",
+    "omni_sparse_mla_combine",
     "omni_sparse_mla_validate", "omni_sparse_mla_resolve_rows",
     "omni_sparse_mla_host_staging_bytes", "omni_sparse_mla_decode_host",
     "omni_sparse_mla_set_profile_events", "omni_sparse_mla_decode_static",
@@ -81,6 +82,8 @@ def load() -> ctypes.CDLL:
     lib.omni_sparse_mla_workspace_bytes.argtypes = [dp]
     lib.omni_sparse_mla_decode.restype = ctypes.c_int
     lib.omni_sparse_mla_decode.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
+    lib.omni_sparse_mla_decode_sink_recent.restype = ctypes.c_int
+    lib.omni_sparse_mla_decode_sink_recent.argtypes = [dp, vp, vp, vp, vp, i32, i32, vp, vp, vp, sz, vp, vp]
     lib.omni_sparse_mla_combine.restype = ctypes.c_int
     lib.omni_sparse_mla_combine.argtypes = [dp, i32, vp, vp, vp, vp, vp, vp]
     lib.omni_sparse_mla_validate.restype = ctypes.c_int
@@ -171,6 +174,22 @@ def omni_sparse_mla_decode(desc, q, kv_cache, page_table, sel_idx, sel_len, out,
         None if workspace is None else ctypes.c_void_p(workspace.data_ptr()), ws_bytes,
         _ptr(device_status, torch.int32, "cuda", "device_status"), _stream(stream))
     _check(code, "omni_sparse_mla_decode")
+
+
+def omni_sparse_mla_decode_sink_recent(desc, q, kv_cache, page_table, ctx_len, n_sink, n_recent, out, lse,
+                                       workspace=None, device_status=None, stream=None) -> None:
+    """Decode with Eq. 2's selection (attention sink + recent tokens) given as N_sink, N_recent and
+    the context length of every request instead of an index list."""
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    code = load().omni_sparse_mla_decode_sink_recent(
+        ctypes.byref(desc), _ptr(q, torch.bfloat16, "cuda", "q"),
+        _ptr(kv_cache, torch.bfloat16, "cuda", "kv_cache"),
+        _ptr(page_table, torch.int32, "cuda", "page_table"),
+        _ptr(ctx_len, torch.int32, "cuda", "ctx_len"), int(n_sink), int(n_recent),
+        _ptr(out, torch.bfloat16, "cuda", "out"), _ptr(lse, torch.float32, "cuda", "lse"),
+        None if workspace is None else ctypes.c_void_p(workspace.data_ptr()), ws_bytes,
+        _ptr(device_status, torch.int32, "cuda", "device_status"), _stream(stream))
+    _check(code, "omni_sparse_mla_decode_sink_recent")
 
 
 OMNI_STATIC_SCRATCH_BYTES = 32 * 1024 * 1024

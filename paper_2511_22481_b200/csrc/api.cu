@@ -235,17 +235,27 @@ size_t omni_sparse_mla_workspace_bytes(const omni_mla_desc_t *desc)
     return workspace_need(desc, choose_splits(desc, device_info().sm_count));
 }
 
-omni_status_t omni_sparse_mla_decode(const omni_mla_desc_t *desc, const void *q,
-                                     const void *kv_cache, const int32_t *page_table,
-                                     const int32_t *sel_idx, const int32_t *sel_len, void *out,
-                                     float *lse, void *workspace, size_t workspace_bytes,
-                                     int32_t *device_status, void *stream_)
+// Shared by the two decode entry points: the selection is an index list (sel_idx, sel_len) or,
+// with sel_idx == nullptr, Eq. 2's ranges (ctx_len, n_sink, n_recent).
+static omni_status_t decode_impl(const omni_mla_desc_t *desc, const void *q, const void *kv_cache,
+                                 const int32_t *page_table, const int32_t *sel_idx,
+                                 const int32_t *sel_len, const int32_t *ctx_len, int32_t n_sink,
+                                 int32_t n_recent, void *out, float *lse, void *workspace,
+                                 size_t workspace_bytes, int32_t *device_status, void *stream_)
 {
-    if (!desc || !q || !kv_cache || !page_table || !sel_idx || !sel_len || !out || !lse)
-        return OMNI_ERR_NULL;
+    const bool ranges = sel_idx == nullptr;
+    if (!desc || !q || !kv_cache || !page_table || !out || !lse) return OMNI_ERR_NULL;
+    if (ranges ? !ctx_len : !sel_len) return OMNI_ERR_NULL;
     if (!desc_ok(desc)) return OMNI_ERR_SHAPE;
+    if (ranges) {
+        // max_sel bounds the selection size the split plan is made for
+        if (n_sink < 0 || n_recent < 0) return OMNI_ERR_SHAPE;
+        const int64_t longest = (int64_t)desc->max_pages_per_req * kPage;
+        const int64_t bound = ((int64_t)n_sink + n_recent < longest) ? (int64_t)n_sink + n_recent : longest;
+        if ((int64_t)desc->max_sel < bound) return OMNI_ERR_SHAPE;
+    }
     if (!aligned(q, 16) || !aligned(kv_cache, 128) || !aligned(out, 16) || !aligned(lse, 4) ||
-        !aligned(page_table, 4) || !aligned(sel_idx, 4) || !aligned(sel_len, 4))
+        !aligned(page_table, 4) || !aligned(sel_idx, 4) || !aligned(sel_len, 4) || !aligned(ctx_len, 4))
         return OMNI_ERR_ALIGN;
     const DeviceInfo &dev = device_info();
     if (!dev.ok) return OMNI_ERR_CUDA;
@@ -259,7 +269,7 @@ omni_status_t omni_sparse_mla_decode(const omni_mla_desc_t *desc, const void *q,
     }
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
 
-    if (desc->flags & OMNI_FLAG_VALIDATE) {
+    if ((desc->flags & OMNI_FLAG_VALIDATE) && !ranges) {
         omni_status_t st = launch_resolve(desc, page_table, sel_idx, sel_len, nullptr, device_status, stream);
         if (st != OMNI_OK) return st;
     }
@@ -270,6 +280,9 @@ omni_status_t omni_sparse_mla_decode(const omni_mla_desc_t *desc, const void *q,
     p.page_table = page_table;
     p.sel_idx = sel_idx;
     p.sel_len = sel_len;
+    p.ctx_len = ctx_len;
+    p.n_sink = n_sink;
+    p.n_recent = n_recent;
     p.out = static_cast<__nv_bfloat16 *>(out);
     p.lse = lse;
     p.part_out = static_cast<float *>(workspace);
@@ -308,6 +321,28 @@ omni_status_t omni_sparse_mla_decode(const omni_mla_desc_t *desc, const void *q,
         return launch_combine(desc->batch, desc->num_heads, splits, p.part_out, p.part_lse, nullptr,
                               out, lse, stream);
     return OMNI_OK;
+}
+
+omni_status_t omni_sparse_mla_decode(const omni_mla_desc_t *desc, const void *q,
+                                     const void *kv_cache, const int32_t *page_table,
+                                     const int32_t *sel_idx, const int32_t *sel_len, void *out,
+                                     float *lse, void *workspace, size_t workspace_bytes,
+                                     int32_t *device_status, void *stream)
+{
+    if (!sel_idx) return OMNI_ERR_NULL;
+    return decode_impl(desc, q, kv_cache, page_table, sel_idx, sel_len, nullptr, 0, 0, out, lse, workspace,
+                       workspace_bytes, device_status, stream);
+}
+
+omni_status_t omni_sparse_mla_decode_sink_recent(const omni_mla_desc_t *desc, const void *q,
+                                                 const void *kv_cache, const int32_t *page_table,
+                                                 const int32_t *ctx_len, int32_t n_sink,
+                                                 int32_t n_recent, void *out, float *lse,
+                                                 void *workspace, size_t workspace_bytes,
+                                                 int32_t *device_status, void *stream)
+{
+    return decode_impl(desc, q, kv_cache, page_table, nullptr, nullptr, ctx_len, n_sink, n_recent, out, lse,
+                       workspace, workspace_bytes, device_status, stream);
 }
 
 omni_status_t omni_sparse_mla_combine(const omni_mla_desc_t *desc, int32_t max_splits,

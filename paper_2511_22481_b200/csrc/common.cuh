@@ -21,8 +21,10 @@ struct DecodeParams {
     const __nv_bfloat16 *q;        // [B, H, 576]
     const __nv_bfloat16 *kv;       // [num_pages * 64, 576]
     const int32_t *page_table;     // [B, max_pages]
-    const int32_t *sel_idx;        // [B, max_sel]
+    const int32_t *sel_idx;        // [B, max_sel]; null: the selection is Eq. 2's two ranges
     const int32_t *sel_len;        // [B]
+    const int32_t *ctx_len;        // [B] context length in tokens (range selection only)
+    int32_t n_sink, n_recent;      // Eq. 2's N_sink and N_recent (range selection only)
     __nv_bfloat16 *out;            // [B, H, 512]
     float *lse;                    // [B, H]
     float *part_out;               // [B, S, H, 512]  (S > 1 only)
@@ -46,6 +48,51 @@ __device__ __forceinline__ void split_range(int n, int splits, int s, int &begin
     const int per = (granules + splits - 1) / splits;
     begin = min(n, s * per * granule);
     end = min(n, (s + 1) * per * granule);
+}
+
+// The selection of one request: the caller's index list, or the index set of Eq. 2 of the
+// paper (attention sink + recent tokens) kept as two ranges, [0, ns) and [rs, M), so that no
+// index list has to exist in memory.  Position j of the selection is list[j] or, for ranges,
+// j itself below ns and rs + (j - ns) from there on.
+struct Selection {
+    const int32_t *list;   // null for ranges
+    int n;                 // selected tokens
+    int ns, rs;            // ranges only: end of the sink range, start of the recent range
+    bool bad;              // the length breaks the contract (n was set to 0)
+};
+
+__device__ __forceinline__ Selection load_selection(const DecodeParams &p, int b)
+{
+    Selection s;
+    s.bad = false;
+    s.ns = s.rs = 0;
+    if (p.sel_idx != nullptr) {
+        s.list = p.sel_idx + (size_t)b * p.max_sel;
+        s.n = __ldg(p.sel_len + b);
+        if (s.n < 0 || s.n > p.max_sel) {
+            s.bad = true;
+            s.n = 0;
+        }
+    } else {
+        s.list = nullptr;
+        int m = __ldg(p.ctx_len + b);
+        if (m < 0 || (int64_t)m > (int64_t)p.max_pages * kPage) {
+            s.bad = true;
+            m = 0;
+        }
+        // 0-based Eq. 2: [0, N_sink) united with [M - N_recent, M); where the two overlap, the
+        // union without repeats
+        s.ns = min(p.n_sink, m);
+        s.rs = max(s.ns, m - min(p.n_recent, m));
+        s.n = s.ns + (m - s.rs);
+    }
+    return s;
+}
+
+__device__ __forceinline__ int32_t selection_at(const Selection &s, int j)
+{
+    if (s.list != nullptr) return __ldg(s.list + j);
+    return j < s.ns ? j : s.rs + (j - s.ns);
 }
 
 // Logical token position -> physical pool row, or -1 if the entry breaks the index contract.

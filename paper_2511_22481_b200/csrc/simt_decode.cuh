@@ -30,11 +30,9 @@ __global__ void __launch_bounds__(kSimtWarps * 32) simt_decode_kernel(DecodePara
     const int h0 = (hg * kSimtWarps + warp) * kSimtHeadsPerWarp;
     if (h0 >= p.heads) return;
 
-    int n = __ldg(p.sel_len + b);
-    if (n < 0 || n > p.max_sel) {
-        if (threadIdx.x == 0) flag_status(p.status, OMNI_DEV_BAD_INDEX);
-        n = 0;
-    }
+    const Selection selection = load_selection(p, b);
+    const int n = selection.n;
+    if (selection.bad && threadIdx.x == 0) flag_status(p.status, OMNI_DEV_BAD_INDEX);
     int begin, end;
     split_range(n, p.splits, s, begin, end);
 
@@ -58,10 +56,9 @@ __global__ void __launch_bounds__(kSimtWarps * 32) simt_decode_kernel(DecodePara
         for (int i = 0; i < 8; ++i) acc[g][i] = make_float2(0.f, 0.f);
     }
 
-    const int32_t *sel = p.sel_idx + (size_t)b * p.max_sel;
     const int32_t *pt = p.page_table + (size_t)b * p.max_pages;
     for (int j = begin; j < end; ++j) {
-        const int64_t row = resolve_row(pt, __ldg(sel + j), p.max_pages, p.num_pages);
+        const int64_t row = resolve_row(pt, selection_at(selection, j), p.max_pages, p.num_pages);
         if (row < 0) {
             if (lane == 0) flag_status(p.status, OMNI_DEV_BAD_INDEX);
             continue;

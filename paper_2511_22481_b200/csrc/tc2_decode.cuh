@@ -361,12 +361,9 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     // may be scheduled as soon as resources allow; it waits in the same way before it reads.
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    int n = __ldg(p.sel_len + b);
-    bool bad_len = false;
-    if (n < 0 || n > p.max_sel) {
-        bad_len = true;
-        n = 0;
-    }
+    const Selection selection = load_selection(p, b);
+    const int n = selection.n;
+    const bool bad_len = selection.bad;
     int begin, end;
     split_range(n, p.splits, s, begin, end, kC2Tile);
     const int tiles = (end - begin + kC2Tile - 1) / kC2Tile;
@@ -396,7 +393,6 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     OMNI_STAMP(0x01, 0);
     OMNI_SPAN(1);
 
-    const int32_t *sel = p.sel_idx + (size_t)b * p.max_sel;
     const int32_t *pt = p.page_table + (size_t)b * p.max_pages;
 
     // Index pipeline of the producers.  Lane l serves tokens l and l+32 of a tile.  The three
@@ -408,8 +404,8 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     };
     auto stage_tokens = [&](int tile, TileIdx &x) {
         const int j0 = begin + tile * kC2Tile + lane, j1 = j0 + 32;
-        x.t0 = (tile < tiles && j0 < end) ? __ldg(sel + j0) : -1;
-        x.t1 = (tile < tiles && j1 < end) ? __ldg(sel + j1) : -1;
+        x.t0 = (tile < tiles && j0 < end) ? selection_at(selection, j0) : -1;
+        x.t1 = (tile < tiles && j1 < end) ? selection_at(selection, j1) : -1;
     };
     auto stage_pages = [&](TileIdx &x) {
         x.pg0 = (x.t0 >= 0 && x.t0 / kPage < p.max_pages) ? __ldg(pt + x.t0 / kPage) : -1;
@@ -578,7 +574,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
                 const int j0 = begin + t * kC2Tile;
                 int row = -1;
                 if (t < tiles && j0 + kC2Tile <= end) {
-                    const int first = __ldg(sel + j0), last = __ldg(sel + j0 + kC2Tile - 1);
+                    const int first = selection_at(selection, j0), last = selection_at(selection, j0 + kC2Tile - 1);
                     if (first >= 0 && first % kPage == 0 && last == first + kC2Tile - 1 && first / kPage < p.max_pages) {
                         const int pg = __ldg(pt + first / kPage);
                         if (pg >= 0 && (int64_t)pg < p.num_pages) row = pg * kPage;

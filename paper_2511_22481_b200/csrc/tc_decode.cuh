@@ -315,12 +315,9 @@ tc_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constan
     // let a dependent kernel (the split merge) be scheduled as soon as resources allow; it still
     // waits for this grid to finish before it reads anything
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    int n = __ldg(p.sel_len + b);
-    bool bad_len = false;
-    if (n < 0 || n > p.max_sel) {
-        bad_len = true;
-        n = 0;
-    }
+    const Selection selection = load_selection(p, b);
+    const int n = selection.n;
+    const bool bad_len = selection.bad;
     int begin, end;
     split_range(n, p.splits, s, begin, end);
     const int tiles = (end - begin + kTile - 1) / kTile;
@@ -375,7 +372,6 @@ tc_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constan
 
     if (warp == 0) {
         // =========================== producer ===========================================
-        const int32_t *sel = p.sel_idx + (size_t)b * p.max_sel;
         const int32_t *pt = p.page_table + (size_t)b * p.max_pages;
         if (lane == 0) {
             mbar_expect_tx(&ctl->q_full, kTileBytes);
@@ -387,8 +383,8 @@ tc_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constan
         // between a freed stage and the copy that refills it.
         auto fetch = [&](int tile, int &t0, int &t1) {
             const int j0 = begin + tile * kTile + lane, j1 = j0 + 32;
-            t0 = (tile < tiles && j0 < end) ? __ldg(sel + j0) : 0;
-            t1 = (tile < tiles && j1 < end) ? __ldg(sel + j1) : 0;
+            t0 = (tile < tiles && j0 < end) ? selection_at(selection, j0) : 0;
+            t1 = (tile < tiles && j1 < end) ? selection_at(selection, j1) : 0;
         };
         auto lookup = [&](int tile, int t0, int t1, int &row_lo, int &row_hi, uint64_t &mask, bool &contig) {
             const int j0 = begin + tile * kTile + lane, j1 = j0 + 32;

@@ -86,6 +86,26 @@ def test_null_and_misaligned_pointers_are_rejected(lib):
     assert lib.omni_sparse_mla_decode_host(ctypes.byref(d), *([ok] * 7), None, 0, ok, 0, None, None) == 1
 
 
+def test_sink_recent_entry_point_checks_its_arguments(lib):
+    ok = ctypes.c_void_p(4096)
+    i32 = ctypes.c_int32
+    call = lambda d, ptrs, ns, nr: lib.omni_sparse_mla_decode_sink_recent(
+        ctypes.byref(d), ptrs[0], ptrs[1], ptrs[2], ptrs[3], i32(ns), i32(nr), ptrs[4], ptrs[5], ok, 1 << 30, None, None)
+    d = _desc(max_sel=256)                                    # 4 pages of 64 tokens per request
+    for missing in range(6):
+        ptrs = [ok] * 6
+        ptrs[missing] = None
+        assert call(d, ptrs, 64, 64) == 1                     # OMNI_ERR_NULL (ctx_len included)
+    assert call(d, [ok] * 6, -1, 64) == 2 and call(d, [ok] * 6, 64, -1) == 2
+    # max_sel must cover min(n_sink + n_recent, longest context)
+    assert call(_desc(max_sel=127), [ok] * 6, 64, 64) == 2
+    assert call(_desc(max_sel=255), [ok] * 6, 1000, 1000) == 2
+    ptrs = [ok] * 6
+    ptrs[3] = ctypes.c_void_p(4096 + 2)                       # ctx_len must be 4-byte aligned
+    assert call(d, ptrs, 64, 64) == 3
+    assert B.omni_sparse_mla_num_launches(_desc(batch=0)) == 0
+
+
 def test_workspace_grows_with_forced_splits(lib):
     a = B.omni_sparse_mla_workspace_bytes(_desc(num_splits=1))
     b = B.omni_sparse_mla_workspace_bytes(_desc(num_splits=4))

@@ -176,6 +176,71 @@ def test_out_of_range_entries_are_flagged_and_skipped(flags):
     assert int(st.item()) == 0
 
 
+# ------------------------------------------------------------------ Eq. 2 as two ranges
+
+def _sink_recent_case(ctx_tokens, n_sink, n_recent, seed, heads=128):
+    """Requests whose selection is the oracle's Eq. 2 index set, plus their context lengths."""
+    from oracle import selection
+    pages = [max(1, -(-m // 64)) for m in ctx_tokens]
+    sels = [selection.sink_recent(m, n_sink, n_recent) for m in ctx_tokens]
+    w = _custom("sink_recent", seed, heads, pages, sels)
+    # positions at or beyond the context length belong to nobody: make sure they are never used
+    tail = torch.ones(w.num_pages * 64, dtype=torch.bool, device=DEV)
+    pt = w.page_table.cpu().numpy()
+    for b, m in enumerate(ctx_tokens):
+        for lp in range(pages[b]):
+            lo = int(pt[b, lp]) * 64
+            tail[lo:lo + max(0, min(64, m - lp * 64))] = False
+    w.kv_cache.view(-1, 576)[tail] = float("nan")
+    ctx = torch.tensor(ctx_tokens, dtype=torch.int32, device=DEV)
+    return w, ctx
+
+
+def _run_ranges(w, ctx, n_sink, n_recent, flags, num_splits=0):
+    desc = B.make_desc(w.batch, w.heads, w.num_pages, w.max_pages_per_req,
+                       max(1, min(n_sink + n_recent, w.max_pages_per_req * 64)), w.scale,
+                       num_splits=num_splits, flags=flags)
+    out = torch.full((w.batch, w.heads, 512), float("nan"), dtype=torch.bfloat16, device=DEV)
+    lse = torch.full((w.batch, w.heads), float("nan"), dtype=torch.float32, device=DEV)
+    ws = torch.empty(B.omni_sparse_mla_workspace_bytes(desc), dtype=torch.uint8, device=DEV)
+    st = torch.zeros(1, dtype=torch.int32, device=DEV)
+    B.omni_sparse_mla_decode_sink_recent(desc, w.q, w.kv_cache, w.page_table, ctx, n_sink, n_recent,
+                                         out, lse, ws, st)
+    torch.cuda.synchronize()
+    return out, lse, int(st.item())
+
+
+@pytest.mark.parametrize("n_sink,n_recent", [(64, 256), (5, 100), (0, 130), (70, 0), (4096, 4096)])
+def test_sink_recent_ranges_match_oracle_on_the_index_set(flags, n_sink, n_recent):
+    # contexts shorter than, equal to and longer than N_sink + N_recent, ragged ends, empty
+    ctx_tokens = [0, 1, 63, 64, 65, 200, 321, 330, 1000, 1537]
+    w, ctx = _sink_recent_case(ctx_tokens, n_sink, n_recent, seed=60)
+    ref_out, ref_lse, _ = oracle_subset(w)
+    for splits in (0, 1, 2, 3):
+        out, lse, status = _run_ranges(w, ctx, n_sink, n_recent, flags, splits)
+        assert status == 0
+        compare(out.cpu(), lse.cpu(), ref_out, ref_lse, "sink+recent ranges S=%d" % splits)
+        assert torch.all(out[0] == 0) and torch.all(torch.isneginf(lse[0]))
+
+
+def test_sink_recent_ranges_equal_the_list_path_bit_for_bit(flags):
+    ctx_tokens = [4096, 777, 130, 2048]
+    w, ctx = _sink_recent_case(ctx_tokens, 64, 512, seed=61)
+    for splits in (1, 2):
+        plan = run_gpu(w, flags, num_splits=splits)
+        out, lse, status = _run_ranges(w, ctx, 64, 512, flags, splits)
+        assert status == 0
+        assert torch.equal(out, plan.out) and torch.equal(lse, plan.lse)
+
+
+def test_sink_recent_bad_context_length_is_flagged():
+    w, ctx = _sink_recent_case([100, 200], 16, 32, seed=62)
+    ctx[1] = w.max_pages_per_req * 64 + 1
+    out, lse, status = _run_ranges(w, ctx, 16, 32, 0)
+    assert status & B.OMNI_DEV_BAD_INDEX
+    assert torch.all(out[1] == 0) and torch.all(torch.isneginf(lse[1]))
+
+
 # ------------------------------------------------------------------ combine entry point
 
 def test_combine_entry_point_matches_oracle():
