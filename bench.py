@@ -153,7 +153,9 @@ def _oracle_sample(w, target_s=15.0, max_requests=None):
 
 
 WORKLOAD_HELP = ("config2 (default, the named benchmark) | config1 | config3 | config4 | "
-                 "config5:<batch>:<selected>[:dense] (one sweep cell)")
+                 "config5:<batch>:<selected>[:dense] (one sweep cell) | "
+                 "eq2:<batch>:<n_sink>:<n_recent>[:list] (the paper's sink + recent rule on 32768-token contexts, "
+                 "through the range entry point, or with :list through the index-list entry point)")
 
 
 def make_workload(spec, dev, batch):
@@ -177,6 +179,12 @@ def make_workload(spec, dev, batch):
         w = W.config5_cell(int(f[1]), int(f[2]), dev, dense_variant=(len(f) > 3 and f[3] == "dense"))
         text = "config5 sweep cell: batch %s, %s tokens/request of ctx 65536, 128 heads" % (
             f[1], "all 65536" if len(f) > 3 else f[2])
+    elif spec.startswith("eq2:"):
+        f = spec.split(":")
+        w = W.sink_recent("eq2", 30, int(f[1]), 128, 32768, int(f[2]), int(f[3]), dev)
+        w.meta["entry"] = "list" if (len(f) > 4 and f[4] == "list") else "ranges"
+        text = ("Eq. 2 selection: batch %s, 128 heads, ctx 32768, N_sink %s + N_recent %s, %s entry point, seed 30"
+                % (f[1], f[2], f[3], "index-list" if w.meta["entry"] == "list" else "range"))
     else:
         raise SystemExit("unknown --workload %r; choose %s" % (spec, WORKLOAD_HELP))
     return w, text
@@ -235,11 +243,19 @@ def main():
     flops = w.selected_tokens * w.heads * FLOP_PER_TOKEN_HEAD
     launches_per_step = B.omni_sparse_mla_num_launches(plan.desc)
 
+    ranges = w.meta.get("entry") == "ranges"
+    ctx_dev = torch.as_tensor(w.ctx_len, dtype=torch.int32).to(dev) if ranges else None
+
     def step(i, ev=None):
         if ev is not None:
             B.omni_sparse_mla_set_profile_events(ev[0], ev[1])
-        B.omni_sparse_mla_decode(plan.desc, w.q, pools[i % clones], w.page_table, w.sel_idx,
-                                 w.sel_len, plan.out, plan.lse, plan.workspace, plan.status)
+        if ranges:
+            B.omni_sparse_mla_decode_sink_recent(plan.desc, w.q, pools[i % clones], w.page_table, ctx_dev,
+                                                 w.meta["n_sink"], w.meta["n_recent"], plan.out, plan.lse,
+                                                 plan.workspace, plan.status)
+        else:
+            B.omni_sparse_mla_decode(plan.desc, w.q, pools[i % clones], w.page_table, w.sel_idx,
+                                     w.sel_len, plan.out, plan.lse, plan.workspace, plan.status)
 
     def barrier():
         torch.cuda.synchronize()

@@ -145,6 +145,28 @@ def page_sparse(name: str, seed: int, batch: int, heads: int, ctx_pages, recent_
                  dict(kind="page_sparse"), make_values)
 
 
+def sink_recent(name: str, seed: int, batch: int, heads: int, ctx_tokens, n_sink: int,
+                n_recent: int, device="cpu", shuffle: bool = True, make_values=True) -> Workload:
+    """The paper's own selection rule (Eq. 2): the first ``n_sink`` and the last ``n_recent``
+    positions of each context, as an increasing list without repeats.  ``ctx_tokens`` is an int
+    or a per-request sequence of context lengths in tokens (they need not fill their last page).
+    The same requests can be given to the range entry point as (ctx_len, n_sink, n_recent):
+    ``meta`` carries the two sizes and ``ctx_len`` the lengths."""
+    rng = np.random.default_rng(seed)
+    ctx = [int(ctx_tokens)] * batch if np.isscalar(ctx_tokens) else [int(x) for x in ctx_tokens]
+    pages = [max(1, -(-m // PAGE)) for m in ctx]
+    tables = _shuffled_tables(rng, pages, shuffle)
+    sels = []
+    for m in ctx:
+        head = np.arange(0, min(n_sink, m))
+        tail = np.arange(max(len(head), m - n_recent), m)
+        sels.append(np.concatenate([head, tail]).astype(np.int32))
+    w = _pack(name, seed, heads, pages, tables, sels, device,
+              dict(kind="sink_recent", n_sink=int(n_sink), n_recent=int(n_recent)), make_values)
+    w.ctx_len = np.asarray(ctx, dtype=np.int64)
+    return w
+
+
 def token_topk(name: str, seed: int, batch: int, heads: int, ctx_pages: int, k: int,
                device="cpu", make_values=True) -> Workload:
     """Token-level selection: the k best positions of a seeded random score vector, in

@@ -72,3 +72,14 @@ def test_same_seed_same_bits():
     import torch
     assert torch.equal(a.q, b.q) and torch.equal(a.kv_cache, b.kv_cache)
     assert torch.equal(a.sel_idx, b.sel_idx)
+
+
+def test_sink_recent_generator_matches_the_oracle_index_set():
+    from oracle import selection
+    ctx = [0, 1, 63, 64, 65, 200, 1000]
+    for n_sink, n_recent in ((64, 256), (5, 100), (0, 130), (70, 0), (4096, 4096)):
+        w = W.sink_recent("t", 3, len(ctx), 2, ctx, n_sink, n_recent, "cpu", make_values=False)
+        for b, m in enumerate(ctx):
+            want = selection.sink_recent(m, n_sink, n_recent)
+            got = w.sel_idx[b, : int(w.sel_len[b])].numpy()
+            assert np.array_equal(got, want)
