@@ -147,6 +147,81 @@ __device__ __forceinline__ void tma_gather4_pair(uint32_t dst, const CUtensorMap
         : "memory");
 }
 
+// Row gathers without the copy engine.  A 4-row TMA gather moves 512 bytes per instruction and
+// the engine takes ~60 clocks for each, which bounds token-level selections; a warp-wide 16-byte
+// cp.async moves the same 512 bytes (four rows x 128 B, eight lanes per row) through the load/store
+// path at several times that rate.  The lanes place their chunks in the 128-byte-swizzled operand
+// layout themselves, and the warp credits the bytes to the stage's barrier with an explicit
+// complete_tx once its copies have landed, exactly as a TMA copy would have.
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int kPending>
+__device__ __forceinline__ void cp_async_wait()
+{
+    asm volatile("cp.async.wait_group %0;" ::"n"(kPending) : "memory");
+}
+// All lanes: wait for this lane's copies of the stage (all but the `newer` most recent groups),
+// make them visible to the tensor core's proxy, then lane 0 credits `bytes` to the barrier.
+__device__ __noinline__ void retire_gathered_stage(uint32_t bar_cluster_addr, uint32_t bytes, bool newer_in_flight,
+                                                      int lane)
+{
+    if (newer_in_flight)
+        cp_async_wait<1>();
+    else
+        cp_async_wait<0>();
+    fence_async_smem();
+    __syncwarp();
+    if (lane == 0) {
+        // The rows are in this CTA's shared memory (wait_group returned in every lane, the proxy
+        // fence and the warp barrier order them before this point) and it is this CTA's own
+        // tensor core that will read them, so a CTA-scope fence is what orders them before the
+        // credit.  A cluster-scope fence here would also wait for the next tile's copies and the
+        // index loads this lane has in flight: measured at ~0.9 us per tile.
+        asm volatile("fence.acq_rel.cta;" ::: "memory");
+        asm volatile("mbarrier.complete_tx.relaxed.cluster.shared::cluster.b64 [%0], %1;" ::"r"(bar_cluster_addr), "r"(bytes)
+                     : "memory");
+    }
+}
+
+// The two gathers are kept out of line so that the producers' loops stay as small as they are
+// for selections that never need them.
+// K role: 32 rows x 9 panels; eight lanes per row, four rows per instruction; chunk c of row r
+// lands at chunk c ^ (r % 8) of its 128-byte line.
+__device__ __noinline__ void gather_k_rows(uint32_t dst, const char *kv_bytes, int own_row, int lane)
+{
+    const int ch = lane & 7;
+#pragma unroll
+    for (int g = 0; g < 8; ++g) {
+        const int r = 4 * g + (lane >> 3);
+        const int src_row = __shfl_sync(0xffffffffu, own_row, r);
+        const char *src = kv_bytes + (size_t)src_row * (kDqk * 2) + ch * 16;
+        const uint32_t d = dst + r * 128 + ((ch ^ (r & 7)) << 4);
+#pragma unroll
+        for (int c = 0; c < kPanels; ++c) cp_async16(d + c * (32 * 128), src + c * 128);
+    }
+    cp_async_commit();
+}
+
+// V role: 64 rows x the four panels of this CTA's value columns (`kv_cols` points at the first).
+__device__ __noinline__ void gather_v_rows(uint32_t dst, const char *kv_cols, int row_lo, int row_hi, int lane)
+{
+    const int ch = lane & 7;
+#pragma unroll
+    for (int g = 0; g < 16; ++g) {
+        const int r = 4 * g + (lane >> 3);
+        const int a = __shfl_sync(0xffffffffu, row_lo, r & 31), c2 = __shfl_sync(0xffffffffu, row_hi, r & 31);
+        const int src_row = r < 32 ? a : c2;
+        const char *src = kv_cols + (size_t)src_row * (kDqk * 2) + ch * 16;
+        const uint32_t d = dst + r * 128 + ((ch ^ (r & 7)) << 4);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) cp_async16(d + c * kPanelBytes, src + c * 128);
+    }
+    cp_async_commit();
+}
+
 // Pair MMA executed by a whole converged warp: one elected lane issues the instruction.  The
 // descriptors arrive as 32-bit halves so that stepping through a tile is a 32-bit add.
 template <bool kAccumulate>
@@ -465,6 +540,8 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
             stage_rows(0, x0, row_lo, row_hi, mask, contig, contig_lo, contig_hi, any_bad);
         }
         bool ok = true;
+        int pending = -1;                    // stage of a gathered tile whose bytes are not credited yet
+        const char *kv_bytes = reinterpret_cast<const char *>(p.kv);
         for (int i = 0; ok && i < tiles; ++i) {
             const int st = i & 1;
             if (lane == 0) {
@@ -481,25 +558,27 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
             OMNI_STAMP(0x10, i);
             const uint32_t dst = smem_base + kC2SmemK + st * kC2KBytes;
             const int own_row = rank ? row_hi : row_lo;
+            bool gathered = false;
             if (rank ? contig_hi : contig_lo) {
                 if (lane == 0) tma_box3d_pair(dst, &kv_k_map, bar, own_row, 0);
             } else {
-                // lane g < 8 gathers tokens 4g..4g+3 of this CTA's 32 into rows 4g..4g+3 of every panel
-                int r[4];
-#pragma unroll
-                for (int k = 0; k < 4; ++k) r[k] = __shfl_sync(0xffffffffu, own_row, (4 * lane + k) & 31);
-                if (lane < 8) {
-#pragma unroll
-                    for (int c = 0; c < kPanels; ++c)
-                        tma_gather4_pair(dst + c * kC2KPanel + lane * 512, &kv_map, bar, c * 64, r[0], r[1], r[2], r[3]);
-                }
+                // scattered rows: eight lanes per row, four rows per instruction, chunk c of row r
+                // lands at chunk c ^ (r % 8) of its 128-byte line
+                gathered = true;
+                gather_k_rows(dst, kv_bytes, own_row, lane);
             }
+            if (pending >= 0) {
+                retire_gathered_stage(map_to_rank(smem_u32(&ctl->k_full[pending]), leader), kC2KBytes, gathered, lane);
+                pending = -1;
+            }
+            if (gathered) pending = st;
             // advance the index pipeline: rows of tile i+1, page ids of tile i+2, positions of tile i+3
             if (i + 1 < tiles) stage_rows(i + 1, x1, row_lo, row_hi, mask, contig, contig_lo, contig_hi, any_bad);
             x1 = x2;
             stage_pages(x1);
             stage_tokens(i + 3, x2);
         }
+        if (pending >= 0) retire_gathered_stage(map_to_rank(smem_u32(&ctl->k_full[pending]), leader), kC2KBytes, false, lane);
         if (lane == 0) *const_cast<volatile int32_t *>(&ctl->k_progress) = 0x7fffffff;
         if (!ok && lane == 0) {
             flag_status(p.status, OMNI_DEV_TIMEOUT | OMNI_DEV_ROLE_PRODUCER_K);
@@ -526,6 +605,8 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
             stage_rows(0, x0, row_lo, row_hi, mask_unused, contig, contig_lo, contig_hi, any_bad);
         }
         bool ok = true;
+        int pending = -1;                    // stage of a gathered tile whose bytes are not credited yet
+        const char *kv_bytes = reinterpret_cast<const char *>(p.kv);
         for (int i = 0; ok && i < tiles; ++i) {
             const int st = i & 1;
             if (i >= 2) ok = mbar_wait(&ctl->pv_done[st], ((i >> 1) - 1) & 1);
@@ -536,29 +617,25 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
             __syncwarp();
             OMNI_STAMP(0x50, i);
             const uint32_t dst = smem_base + kC2SmemV + st * kC2VBytes;
+            bool gathered = false;
             if (contig) {
                 if (lane == 0) tma_box3d_pair(dst, &kv_v_map, bar, row_lo, 4 * (int)rank);
             } else {
-                // lane g < 16 gathers tokens 4g..4g+3 into rows 4g..4g+3 of the four panels
-                int r[4];
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const int src = (4 * lane + k) & 31;
-                    const int a = __shfl_sync(0xffffffffu, row_lo, src), c = __shfl_sync(0xffffffffu, row_hi, src);
-                    r[k] = lane < 8 ? a : c;
-                }
-                if (lane < 16) {
-#pragma unroll
-                    for (int c = 0; c < 4; ++c)
-                        tma_gather4_pair(dst + c * kPanelBytes + lane * 512, &kv_map, bar, ((int)rank * 4 + c) * 64, r[0],
-                                         r[1], r[2], r[3]);
-                }
+                // scattered rows: the four panels of this CTA's value columns, 64 tokens
+                gathered = true;
+                gather_v_rows(dst, kv_bytes + (int)rank * 512, row_lo, row_hi, lane);
             }
+            if (pending >= 0) {
+                retire_gathered_stage(map_to_rank(smem_u32(&ctl->v_full[pending]), leader), kC2VBytes, gathered, lane);
+                pending = -1;
+            }
+            if (gathered) pending = st;
             if (i + 1 < tiles) stage_rows(i + 1, x1, row_lo, row_hi, mask_unused, contig, contig_lo, contig_hi, any_bad);
             x1 = x2;
             stage_pages(x1);
             stage_tokens(i + 3, x2);
         }
+        if (pending >= 0) retire_gathered_stage(map_to_rank(smem_u32(&ctl->v_full[pending]), leader), kC2VBytes, false, lane);
         if (!ok && lane == 0) {
             flag_status(p.status, OMNI_DEV_TIMEOUT | OMNI_DEV_ROLE_PRODUCER_V);
             *abort_flag = 1;
