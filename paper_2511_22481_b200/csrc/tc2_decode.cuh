@@ -761,9 +761,21 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
             using I1 = std::integral_constant<int, 1>;
             using I2 = std::integral_constant<int, 2>;
             // step j of a group of six tiles: Q K^T of tile i+2 (stage i & 1, buffer (i+2) % 3), then P V of tile i
+            // (if the K rows of tile i+2 have not landed yet while P and V of tile i are ready, P V goes first)
             auto step = [&](auto kpar_tag, auto sbuf_tag, int i) -> bool {
-                if (i + 2 < tiles_u && !qk_tile(kpar_tag, sbuf_tag, i + 2)) return false;
-                return pv_tile(kpar_tag, i);
+                constexpr int kpar = decltype(kpar_tag)::value;
+                bool qk_todo = i + 2 < tiles_u;
+                if (qk_todo) {
+                    const bool k_ready = __all_sync(0xffffffffu, mbar_test(&ctl->k_full[kpar], ((i + 2) >> 1) & 1));
+                    const bool pv_ready = __all_sync(0xffffffffu, mbar_test(&ctl->p_full[kpar], (i >> 1) & 1) &&
+                                                                      mbar_test(&ctl->v_full[kpar], (i >> 1) & 1));
+                    if (k_ready || !pv_ready) {
+                        if (!qk_tile(kpar_tag, sbuf_tag, i + 2)) return false;
+                        qk_todo = false;
+                    }
+                }
+                if (!pv_tile(kpar_tag, i)) return false;
+                return !qk_todo || qk_tile(kpar_tag, sbuf_tag, i + 2);
             };
             bool ok = mbar_wait(&ctl->q_full, 0);
             ok = __all_sync(0xffffffffu, ok);
