@@ -1,0 +1,65 @@
+"""A layer loop under one CUDA graph: the paper applies its compression per layer with a 0/1
+pattern (sparse sink + recent selection on some layers, the full context on the others).  Here a
+few "layers" (each with its own q and its own pattern bit) are captured into one CUDA graph
+through the public entry points and replayed; every layer's result must equal, bit for bit, what
+the same calls produce when launched one by one."""
+import pytest
+import torch
+
+from paper_2511_22481_b200 import binding as B
+from paper_2511_22481_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _layer_inputs(w, layers, seed):
+    g = torch.Generator(device=DEV).manual_seed(seed)
+    return [(0.5 * torch.randn(w.q.shape, generator=g, device=DEV, dtype=torch.float32)).to(torch.bfloat16)
+            for _ in range(layers)]
+
+
+def test_layer_loop_in_one_cuda_graph_matches_eager():
+    pattern = [1, 0, 1, 1, 0]                      # 1: Eq. 2 selection (sink 64 + recent 512), 0: full context
+    ctx_tokens = [4096, 2500, 3333, 4000]
+    sparse = W.sink_recent("layers", 70, len(ctx_tokens), 128, ctx_tokens, 64, 512, DEV)
+    ctx = torch.as_tensor(sparse.ctx_len, dtype=torch.int32).to(DEV)
+    qs = _layer_inputs(sparse, len(pattern), 71)
+    max_ctx = sparse.max_pages_per_req * 64
+
+    def make(max_sel):
+        desc = B.make_desc(sparse.batch, 128, sparse.num_pages, sparse.max_pages_per_req, max_sel, sparse.scale)
+        ws = torch.empty(B.omni_sparse_mla_workspace_bytes(desc), dtype=torch.uint8, device=DEV)
+        return desc, ws
+
+    plans = {1: make(64 + 512), 0: make(max_ctx)}
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+
+    def run_layers(outs, lses):
+        for l, bit in enumerate(pattern):
+            desc, ws = plans[bit]
+            n_sink, n_recent = (64, 512) if bit else (max_ctx, 0)       # N_sink >= M selects the whole context
+            B.omni_sparse_mla_decode_sink_recent(desc, qs[l], sparse.kv_cache, sparse.page_table, ctx,
+                                                 n_sink, n_recent, outs[l], lses[l], ws, status)
+
+    new = lambda: ([torch.empty((sparse.batch, 128, 512), dtype=torch.bfloat16, device=DEV) for _ in pattern],
+                   [torch.empty((sparse.batch, 128), dtype=torch.float32, device=DEV) for _ in pattern])
+    eager_out, eager_lse = new()
+    run_layers(eager_out, eager_lse)               # also the warm-up: attributes and tensor maps are set up here
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+
+    graph_out, graph_lse = new()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        run_layers(graph_out, graph_lse)
+    for o in graph_out:
+        o.zero_()
+    for _ in range(2):
+        graph.replay()
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for l in range(len(pattern)):
+        assert torch.equal(graph_out[l], eager_out[l]) and torch.equal(graph_lse[l], eager_lse[l]), l
+    # the sparse and the dense layers do differ (the pattern is not ignored)
+    assert not torch.equal(eager_out[0], eager_out[1])
