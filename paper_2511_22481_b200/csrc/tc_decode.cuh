@@ -312,8 +312,10 @@ tc_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constan
     const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;  // warp-uniform
     const int h0 = hg * kTcHeads;
 
-    // let a dependent kernel (the split merge) be scheduled as soon as resources allow; it still
-    // waits for this grid to finish before it reads anything
+    // Programmatic dependent launch, both ways: nothing in global memory is touched until the
+    // kernel before this one in the stream has completed, and the kernel after this one (the split
+    // merge) may be scheduled as soon as resources allow; it waits in the same way before it reads.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const Selection selection = load_selection(p, b);
     const int n = selection.n;
@@ -803,8 +805,18 @@ inline omni_status_t launch_tc_decode(const DecodeParams &p, cudaStream_t stream
     if (!make_panel_map(&kv_page_map, p.kv, (uint64_t)p.num_pages * kPage, kTile, kPanels)) return OMNI_ERR_CUDA;
     const int head_groups = (p.heads + kTcHeads - 1) / kTcHeads;
     const unsigned grid = (unsigned)(p.batch * p.splits * head_groups);
-    tc_decode_kernel<<<grid, kTcThreads, kTcSmemBytes, stream>>>(q_map, kv_map, kv_page_map, p);
-    return cudaPeekAtLastError() == cudaSuccess ? OMNI_OK : OMNI_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kTcThreads);
+    cfg.dynamicSmemBytes = kTcSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;    // see the kernel's first lines
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, tc_decode_kernel, q_map, kv_map, kv_page_map, p) == cudaSuccess ? OMNI_OK
+                                                                                                      : OMNI_ERR_CUDA;
 }
 
 }  // namespace omni
