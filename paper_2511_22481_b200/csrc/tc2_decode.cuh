@@ -17,7 +17,7 @@
 // is consumed and Q K^T of tile i+1 overlaps the softmax of tile i.  Every refill is ONE 3-D TMA
 // box {64 columns, rows, panels}: the copy engine sustains only about 4 M instructions/s per SM,
 // so 8 KiB boxes cap an SM near 32 GB/s while 32-72 KiB boxes reach 90-150 GB/s.  Tiles that are
-// not 64 consecutive pool rows fall back to 4-row gathers.
+// not 64 consecutive pool rows are gathered row by row with cp.async (see below).
 //
 // All MMAs are issued by warp 1 of CTA 0 in "whatever is ready" order: the whole warp runs the
 // loop with warp-uniform control flow and one elected lane issues each instruction (a lone
@@ -134,16 +134,6 @@ __device__ __forceinline__ void tma_box3d_pair(uint32_t dst, const CUtensorMap *
         "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
         " [%0], [%1, {%2, %3, %4}], [%5];"
         ::"r"(dst), "l"(map), "r"(0), "r"(row), "r"(panel), "r"(bar_cluster_addr)
-        : "memory");
-}
-
-__device__ __forceinline__ void tma_gather4_pair(uint32_t dst, const CUtensorMap *map, uint32_t bar_cluster_addr,
-                                                 int col, int r0, int r1, int r2, int r3)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes"
-        " [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
-        ::"r"(dst), "l"(map), "r"(col), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(bar_cluster_addr)
         : "memory");
 }
 
@@ -367,7 +357,7 @@ __device__ __forceinline__ void cluster_merge_exchange(const DecodeParams &p, C2
 }
 
 __global__ void __launch_bounds__(kC2Threads, 1)
-tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap kv_map,
+tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
                   const __grid_constant__ CUtensorMap kv_k_map, const __grid_constant__ CUtensorMap kv_v_map,
                   const __grid_constant__ CUtensorMap kv_tile_map, DecodeParams p)
 {
@@ -1099,10 +1089,9 @@ inline omni_status_t launch_tc2_decode(const DecodeParams &p, cudaStream_t strea
             return OMNI_ERR_CUDA;
         attr_set[dev] = true;
     }
-    CUtensorMap q_map, kv_map, kv_k_map, kv_v_map, kv_tile_map;
+    CUtensorMap q_map, kv_k_map, kv_v_map, kv_tile_map;
     if (!make_panel_map(&kv_tile_map, p.kv, (uint64_t)p.num_pages * kPage, kTile, kPanels)) return OMNI_ERR_CUDA;
     if (!make_panel_map(&q_map, p.q, (uint64_t)p.batch * p.heads, kTcHeads, kPanels)) return OMNI_ERR_CUDA;
-    if (!make_row_map(&kv_map, p.kv, (uint64_t)p.num_pages * kPage, 1)) return OMNI_ERR_CUDA;
     if (!make_panel_map(&kv_k_map, p.kv, (uint64_t)p.num_pages * kPage, 32, kPanels)) return OMNI_ERR_CUDA;
     if (!make_panel_map(&kv_v_map, p.kv, (uint64_t)p.num_pages * kPage, kTile, 4)) return OMNI_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
@@ -1121,7 +1110,7 @@ inline omni_status_t launch_tc2_decode(const DecodeParams &p, cudaStream_t strea
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, tc2_decode_kernel, q_map, kv_map, kv_k_map, kv_v_map, kv_tile_map, p) == cudaSuccess
+    return cudaLaunchKernelEx(&cfg, tc2_decode_kernel, q_map, kv_k_map, kv_v_map, kv_tile_map, p) == cudaSuccess
                ? OMNI_OK
                : OMNI_ERR_CUDA;
 }

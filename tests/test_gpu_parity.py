@@ -56,7 +56,8 @@ def test_ragged_lengths_and_tails(flags):
 @pytest.mark.parametrize("heads", [1, 16, 48, 64, 80, 128])
 def test_head_counts(flags, heads):
     w = W.token_topk("heads%d" % heads, 42, 2, heads, 8, 200, DEV)
-    check_workload(w, flags, what="H=%d" % heads)
+    for splits in (0, 2, 3):                 # 2: merged inside a cluster when the pair kernel runs
+        check_workload(w, flags, num_splits=splits, what="H=%d S=%d" % (heads, splits))
 
 
 def test_token_level_unsorted_selection(flags):
