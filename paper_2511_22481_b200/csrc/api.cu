@@ -294,6 +294,11 @@ static omni_status_t decode_impl(const omni_mla_desc_t *desc, const void *q, con
     // Two splits of a request can be merged inside a cluster of two CTA pairs, without partial
     // results in global memory, as long as all those clusters are resident at once.
     if (merge_in_cluster(desc, splits)) p.cluster_merge = 1;
+    // several waves of work units: start the longest requests first (the kernel ranks them itself)
+    p.longest_first = (use_pair_kernel(desc) && !p.cluster_merge && desc->batch <= 256 &&
+                       (long)desc->batch * splits > dev.sm_count / 2)
+                          ? 1
+                          : 0;
     if (splits > 1 && merge_in_kernel(desc)) {
         p.counters = reinterpret_cast<int32_t *>(static_cast<char *>(workspace) + part_out_bytes(desc, splits) +
                                                  part_lse_bytes(desc, splits));
@@ -388,7 +393,7 @@ int omni_trace_read(void *host, size_t bytes)
 }
 int omni_span_read(void *host, size_t bytes)
 {
-    if (bytes > sizeof(unsigned long long) * 2048 * 4) return 1;
+    if (bytes > sizeof(unsigned long long) * 2048 * 8) return 1;
     return cudaMemcpyFromSymbol(host, g_span, bytes) == cudaSuccess ? 0 : 2;
 }
 int omni_trace_clear(void)

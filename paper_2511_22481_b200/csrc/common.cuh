@@ -35,6 +35,7 @@ struct DecodeParams {
     int64_t num_pages;
     int32_t batch, heads, max_pages, max_sel, splits;
     int32_t cluster_merge;         // 1: two splits, merged inside a cluster of two CTA pairs
+    int32_t longest_first;         // 1: work units take the requests in order of decreasing selection size
     float scale_log2;              // softmax_scale * log2(e)
 };
 
@@ -124,7 +125,7 @@ __device__ __forceinline__ unsigned long long trace_time_ns()
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-__device__ unsigned long long g_span[2048][4];   // per CTA: entry, set-up done, last P V retired, exit
+__device__ unsigned long long g_span[2048][8];   // per CTA: entry, set-up done, last P V retired, exit, merge phases
 #define OMNI_SPAN(slot)                                                                             \
     do {                                                                                            \
         if (threadIdx.x == 64 && blockIdx.x < 2048) g_span[blockIdx.x][slot] = trace_time_ns();     \

@@ -379,7 +379,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
 
     const int pair = blockIdx.x >> 1;
     const int s = p.cluster_merge ? (int)(crank >> 1) : pair % p.splits;
-    const int b = p.cluster_merge ? (int)(blockIdx.x >> 2) : pair / p.splits;
+    int b = p.cluster_merge ? (int)(blockIdx.x >> 2) : pair / p.splits;
     const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;  // warp-uniform
     const int h0 = (int)rank * kTcHeads;
     const int head_rows = min(kTcHeads, p.heads - h0);
@@ -426,6 +426,25 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
     // may be scheduled as soon as resources allow; it waits in the same way before it reads.
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (p.longest_first) {
+        // The grid runs in several waves and CTAs start in index order, so the requests are
+        // taken longest first (ties by index): a long request that started last would otherwise
+        // run on alone at the end.  Every CTA ranks the (at most 256) selection sizes itself:
+        // request j has rank #{i : n_i > n_j, or n_i = n_j and i < j}, and this pair takes the
+        // request whose rank is its own place in the grid.
+        int *lens = reinterpret_cast<int *>(smem);               // operand tiles are not in use yet
+        for (int j = threadIdx.x; j < p.batch; j += kC2Threads) lens[j] = load_selection(p, j).n;
+        __syncthreads();
+        for (int j = threadIdx.x; j < p.batch; j += kC2Threads) {
+            const int nj = lens[j];
+            int before = 0;
+            for (int i = 0; i < p.batch; ++i) before += (lens[i] > nj) || (lens[i] == nj && i < j);
+            if (before == b) ctl->merge_flag = (uint32_t)j;
+        }
+        __syncthreads();
+        b = (int)ctl->merge_flag;
+        __syncthreads();                                          // smem is handed to the producers next
+    }
     const Selection selection = load_selection(p, b);
     const int n = selection.n;
     const bool bad_len = selection.bad;
