@@ -162,6 +162,40 @@ omni_status_t omni_sparse_mla_decode_sink_recent(const omni_mla_desc_t *desc, co
                                                  int32_t *device_status, void *stream);
 
 /*
+ * Rolling cache of a compressed layer (the paper's layer-wise KV-cache compression: a layer
+ * whose pattern bit is 1 only ever attends to the index set of Eq. 2, so it needs to store
+ * nothing but the attention sink and the recent window).  Per request such a layer owns
+ * omni_rolling_pages_per_request(n_sink, n_recent) = ceil(N_sink/64) + ceil(N_recent/64) + 1
+ * pages, listed in its page_table row: the first ceil(N_sink/64) hold positions
+ * [0, 64*ceil(N_sink/64)) for good, the others are reused round-robin by all later 64-token
+ * blocks of the context.  The token at absolute position t is therefore found at position
+ *     t                                                     if t / 64 < sink_pages
+ *     (sink_pages + (t/64 - sink_pages) % ring_pages)*64 + t%64   otherwise
+ * of that short page table, whatever the context length.
+ *
+ * omni_kv_append_rolling writes one new latent row per request: new_rows[b] (bf16 [B, 576],
+ * 16-byte aligned) becomes the token at position ctx_len[b] (the length BEFORE the append; the
+ * caller advances its own counter afterwards) and overwrites the oldest block's slot once the
+ * ring has gone round.  A negative length or a bad page id sets OMNI_DEV_BAD_INDEX and skips
+ * the request.  desc supplies batch, num_pages and max_pages_per_req (>= the pages per request
+ * above, else OMNI_ERR_SHAPE).
+ *
+ * omni_sparse_mla_decode_rolling is omni_sparse_mla_decode_sink_recent over that layout: the
+ * same index set, the same result bit for bit as on an uncompressed cache holding the same
+ * rows, for any ctx_len[b] >= 0.  desc->max_sel must be at least n_sink + n_recent.
+ */
+int32_t omni_rolling_pages_per_request(int32_t n_sink, int32_t n_recent);
+omni_status_t omni_kv_append_rolling(const omni_mla_desc_t *desc, void *kv_cache,
+                                     const int32_t *page_table, const int32_t *ctx_len,
+                                     const void *new_rows, int32_t n_sink, int32_t n_recent,
+                                     int32_t *device_status, void *stream);
+omni_status_t omni_sparse_mla_decode_rolling(const omni_mla_desc_t *desc, const void *q,
+                                             const void *kv_cache, const int32_t *page_table,
+                                             const int32_t *ctx_len, int32_t n_sink, int32_t n_recent,
+                                             void *out, float *lse, void *workspace,
+                                             size_t workspace_bytes, int32_t *device_status, void *stream);
+
+/*
  * Merge of split-KV partial results (the step that follows a partition of M into disjoint
  * ranges; Eq. 1 is recovered exactly because softmax normalisers add):
  *     lse[b,h]   = ln sum_s exp(part_lse[b,s,h])

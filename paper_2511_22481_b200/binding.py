@@ -27,6 +27,7 @@ OMNI_FLAG_NO_CLUSTER_MERGE = 8
 EXPORTS = (
     "omni_version", "omni_status_string", "omni_sparse_mla_num_splits", "omni_sparse_mla_num_launches",
     "omni_sparse_mla_workspace_bytes", "omni_sparse_mla_decode", "omni_sparse_mla_decode_sink_recent",
+    "omni_rolling_pages_per_request", "omni_kv_append_rolling", "omni_sparse_mla_decode_rolling",
     "omni_sparse_mla_combine",
     "omni_sparse_mla_validate", "omni_sparse_mla_resolve_rows",
     "omni_sparse_mla_host_staging_bytes", "omni_sparse_mla_decode_host",
@@ -84,6 +85,12 @@ def load() -> ctypes.CDLL:
     lib.omni_sparse_mla_decode.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
     lib.omni_sparse_mla_decode_sink_recent.restype = ctypes.c_int
     lib.omni_sparse_mla_decode_sink_recent.argtypes = [dp, vp, vp, vp, vp, i32, i32, vp, vp, vp, sz, vp, vp]
+    lib.omni_sparse_mla_decode_rolling.restype = ctypes.c_int
+    lib.omni_sparse_mla_decode_rolling.argtypes = [dp, vp, vp, vp, vp, i32, i32, vp, vp, vp, sz, vp, vp]
+    lib.omni_kv_append_rolling.restype = ctypes.c_int
+    lib.omni_kv_append_rolling.argtypes = [dp, vp, vp, vp, vp, i32, i32, vp, vp]
+    lib.omni_rolling_pages_per_request.restype = i32
+    lib.omni_rolling_pages_per_request.argtypes = [i32, i32]
     lib.omni_sparse_mla_combine.restype = ctypes.c_int
     lib.omni_sparse_mla_combine.argtypes = [dp, i32, vp, vp, vp, vp, vp, vp]
     lib.omni_sparse_mla_validate.restype = ctypes.c_int
@@ -190,6 +197,36 @@ def omni_sparse_mla_decode_sink_recent(desc, q, kv_cache, page_table, ctx_len, n
         None if workspace is None else ctypes.c_void_p(workspace.data_ptr()), ws_bytes,
         _ptr(device_status, torch.int32, "cuda", "device_status"), _stream(stream))
     _check(code, "omni_sparse_mla_decode_sink_recent")
+
+
+def omni_rolling_pages_per_request(n_sink: int, n_recent: int) -> int:
+    return int(load().omni_rolling_pages_per_request(int(n_sink), int(n_recent)))
+
+
+def omni_kv_append_rolling(desc, kv_cache, page_table, ctx_len, new_rows, n_sink, n_recent,
+                           device_status=None, stream=None) -> None:
+    """Append one latent row per request to the rolling cache of a compressed layer."""
+    code = load().omni_kv_append_rolling(
+        ctypes.byref(desc), _ptr(kv_cache, torch.bfloat16, "cuda", "kv_cache"),
+        _ptr(page_table, torch.int32, "cuda", "page_table"), _ptr(ctx_len, torch.int32, "cuda", "ctx_len"),
+        _ptr(new_rows, torch.bfloat16, "cuda", "new_rows"), int(n_sink), int(n_recent),
+        _ptr(device_status, torch.int32, "cuda", "device_status"), _stream(stream))
+    _check(code, "omni_kv_append_rolling")
+
+
+def omni_sparse_mla_decode_rolling(desc, q, kv_cache, page_table, ctx_len, n_sink, n_recent, out, lse,
+                                   workspace=None, device_status=None, stream=None) -> None:
+    """Decode over the rolling cache of a compressed layer (Eq. 2's index set, any context length)."""
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    code = load().omni_sparse_mla_decode_rolling(
+        ctypes.byref(desc), _ptr(q, torch.bfloat16, "cuda", "q"),
+        _ptr(kv_cache, torch.bfloat16, "cuda", "kv_cache"),
+        _ptr(page_table, torch.int32, "cuda", "page_table"),
+        _ptr(ctx_len, torch.int32, "cuda", "ctx_len"), int(n_sink), int(n_recent),
+        _ptr(out, torch.bfloat16, "cuda", "out"), _ptr(lse, torch.float32, "cuda", "lse"),
+        None if workspace is None else ctypes.c_void_p(workspace.data_ptr()), ws_bytes,
+        _ptr(device_status, torch.int32, "cuda", "device_status"), _stream(stream))
+    _check(code, "omni_sparse_mla_decode_rolling")
 
 
 OMNI_STATIC_SCRATCH_BYTES = 32 * 1024 * 1024

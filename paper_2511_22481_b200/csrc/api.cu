@@ -54,6 +54,11 @@ bool desc_ok(const omni_mla_desc_t *d)
            d->max_sel >= 1 && d->num_splits >= 0 && d->num_splits <= kMaxSplits;
 }
 
+// Pages of a compressed layer's rolling cache: the sink pages are kept for good, the ring holds
+// the recent window (which can straddle one more page than it fills).
+int64_t rolling_sink_pages(int32_t n_sink) { return ((int64_t)n_sink + kPage - 1) / kPage; }
+int64_t rolling_ring_pages(int32_t n_recent) { return ((int64_t)n_recent + kPage - 1) / kPage + 1; }
+
 bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
 // More than 64 heads run on the paired-CTA kernel (one cluster of two CTAs per work unit).
@@ -240,7 +245,7 @@ size_t omni_sparse_mla_workspace_bytes(const omni_mla_desc_t *desc)
 static omni_status_t decode_impl(const omni_mla_desc_t *desc, const void *q, const void *kv_cache,
                                  const int32_t *page_table, const int32_t *sel_idx,
                                  const int32_t *sel_len, const int32_t *ctx_len, int32_t n_sink,
-                                 int32_t n_recent, void *out, float *lse, void *workspace,
+                                 int32_t n_recent, bool rolling, void *out, float *lse, void *workspace,
                                  size_t workspace_bytes, int32_t *device_status, void *stream_)
 {
     const bool ranges = sel_idx == nullptr;
@@ -251,8 +256,11 @@ static omni_status_t decode_impl(const omni_mla_desc_t *desc, const void *q, con
         // max_sel bounds the selection size the split plan is made for
         if (n_sink < 0 || n_recent < 0) return OMNI_ERR_SHAPE;
         const int64_t longest = (int64_t)desc->max_pages_per_req * kPage;
-        const int64_t bound = ((int64_t)n_sink + n_recent < longest) ? (int64_t)n_sink + n_recent : longest;
+        // a rolling cache holds contexts of any length, so only N_sink + N_recent bounds the selection
+        const int64_t bound = (rolling || (int64_t)n_sink + n_recent < longest) ? (int64_t)n_sink + n_recent : longest;
         if ((int64_t)desc->max_sel < bound) return OMNI_ERR_SHAPE;
+        if (rolling && (int64_t)desc->max_pages_per_req < rolling_sink_pages(n_sink) + rolling_ring_pages(n_recent))
+            return OMNI_ERR_SHAPE;
     }
     if (!aligned(q, 16) || !aligned(kv_cache, 128) || !aligned(out, 16) || !aligned(lse, 4) ||
         !aligned(page_table, 4) || !aligned(sel_idx, 4) || !aligned(sel_len, 4) || !aligned(ctx_len, 4))
@@ -283,6 +291,8 @@ static omni_status_t decode_impl(const omni_mla_desc_t *desc, const void *q, con
     p.ctx_len = ctx_len;
     p.n_sink = n_sink;
     p.n_recent = n_recent;
+    p.sink_pages = rolling ? (int32_t)rolling_sink_pages(n_sink) : 0;
+    p.ring_pages = rolling ? (int32_t)rolling_ring_pages(n_recent) : 0;
     p.out = static_cast<__nv_bfloat16 *>(out);
     p.lse = lse;
     p.part_out = static_cast<float *>(workspace);
@@ -335,7 +345,7 @@ omni_status_t omni_sparse_mla_decode(const omni_mla_desc_t *desc, const void *q,
                                      int32_t *device_status, void *stream)
 {
     if (!sel_idx) return OMNI_ERR_NULL;
-    return decode_impl(desc, q, kv_cache, page_table, sel_idx, sel_len, nullptr, 0, 0, out, lse, workspace,
+    return decode_impl(desc, q, kv_cache, page_table, sel_idx, sel_len, nullptr, 0, 0, false, out, lse, workspace,
                        workspace_bytes, device_status, stream);
 }
 
@@ -346,8 +356,42 @@ omni_status_t omni_sparse_mla_decode_sink_recent(const omni_mla_desc_t *desc, co
                                                  void *workspace, size_t workspace_bytes,
                                                  int32_t *device_status, void *stream)
 {
-    return decode_impl(desc, q, kv_cache, page_table, nullptr, nullptr, ctx_len, n_sink, n_recent, out, lse,
+    return decode_impl(desc, q, kv_cache, page_table, nullptr, nullptr, ctx_len, n_sink, n_recent, false, out, lse,
                        workspace, workspace_bytes, device_status, stream);
+}
+
+omni_status_t omni_sparse_mla_decode_rolling(const omni_mla_desc_t *desc, const void *q,
+                                             const void *kv_cache, const int32_t *page_table,
+                                             const int32_t *ctx_len, int32_t n_sink, int32_t n_recent,
+                                             void *out, float *lse, void *workspace,
+                                             size_t workspace_bytes, int32_t *device_status, void *stream)
+{
+    return decode_impl(desc, q, kv_cache, page_table, nullptr, nullptr, ctx_len, n_sink, n_recent, true, out, lse,
+                       workspace, workspace_bytes, device_status, stream);
+}
+
+int32_t omni_rolling_pages_per_request(int32_t n_sink, int32_t n_recent)
+{
+    if (n_sink < 0 || n_recent < 0) return 0;
+    const int64_t pages = rolling_sink_pages(n_sink) + rolling_ring_pages(n_recent);
+    return pages > 0x7fffffff ? 0 : (int32_t)pages;
+}
+
+omni_status_t omni_kv_append_rolling(const omni_mla_desc_t *desc, void *kv_cache,
+                                     const int32_t *page_table, const int32_t *ctx_len,
+                                     const void *new_rows, int32_t n_sink, int32_t n_recent,
+                                     int32_t *device_status, void *stream)
+{
+    if (!desc || !kv_cache || !page_table || !ctx_len || !new_rows) return OMNI_ERR_NULL;
+    if (!desc_ok(desc) || n_sink < 0 || n_recent < 0) return OMNI_ERR_SHAPE;
+    if ((int64_t)desc->max_pages_per_req < rolling_sink_pages(n_sink) + rolling_ring_pages(n_recent)) return OMNI_ERR_SHAPE;
+    if (!aligned(kv_cache, 128) || !aligned(new_rows, 16) || !aligned(page_table, 4) || !aligned(ctx_len, 4))
+        return OMNI_ERR_ALIGN;
+    append_rolling_kernel<<<(unsigned)desc->batch, 72, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<__nv_bfloat16 *>(kv_cache), page_table, ctx_len, static_cast<const __nv_bfloat16 *>(new_rows),
+        desc->max_pages_per_req, desc->num_pages, (int)rolling_sink_pages(n_sink), (int)rolling_ring_pages(n_recent),
+        device_status);
+    return cudaPeekAtLastError() == cudaSuccess ? OMNI_OK : OMNI_ERR_CUDA;
 }
 
 omni_status_t omni_sparse_mla_combine(const omni_mla_desc_t *desc, int32_t max_splits,

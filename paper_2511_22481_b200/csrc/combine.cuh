@@ -79,4 +79,30 @@ __global__ void __launch_bounds__(256) resolve_rows_kernel(const int32_t *__rest
     if (bad) flag_status(status, OMNI_DEV_BAD_INDEX);
 }
 
+// Appends one latent row per request to the rolling cache of a compressed layer: the row of the
+// token at absolute position ctx_len[b] goes to rolling_position(ctx_len[b]) of the request's
+// page table.  72 threads per request, 16 bytes each.
+__global__ void __launch_bounds__(72) append_rolling_kernel(__nv_bfloat16 *__restrict__ kv,
+                                                            const int32_t *__restrict__ page_table,
+                                                            const int32_t *__restrict__ ctx_len,
+                                                            const __nv_bfloat16 *__restrict__ new_rows,
+                                                            int max_pages, int64_t num_pages, int sink_pages,
+                                                            int ring_pages, int32_t *status)
+{
+    const int b = blockIdx.x;
+    const int32_t t = __ldg(ctx_len + b);
+    int64_t row = -1;
+    if (t >= 0) {
+        const int32_t pos = rolling_position(t, sink_pages, ring_pages);
+        row = resolve_row(page_table + (size_t)b * max_pages, pos, max_pages, num_pages);
+    }
+    if (row < 0) {
+        if (threadIdx.x == 0) flag_status(status, OMNI_DEV_BAD_INDEX);
+        return;
+    }
+    const uint4 *src = reinterpret_cast<const uint4 *>(new_rows + (size_t)b * kDqk);
+    uint4 *dst = reinterpret_cast<uint4 *>(kv + (size_t)row * kDqk);
+    dst[threadIdx.x] = __ldg(src + threadIdx.x);
+}
+
 }  // namespace omni

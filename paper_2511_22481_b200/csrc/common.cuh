@@ -25,6 +25,7 @@ struct DecodeParams {
     const int32_t *sel_len;        // [B]
     const int32_t *ctx_len;        // [B] context length in tokens (range selection only)
     int32_t n_sink, n_recent;      // Eq. 2's N_sink and N_recent (range selection only)
+    int32_t sink_pages, ring_pages; // rolling cache of a compressed layer (ring_pages > 0), see rolling_position
     __nv_bfloat16 *out;            // [B, H, 512]
     float *lse;                    // [B, H]
     float *part_out;               // [B, S, H, 512]  (S > 1 only)
@@ -51,6 +52,18 @@ __device__ __forceinline__ void split_range(int n, int splits, int s, int &begin
     end = min(n, (s + 1) * per * granule);
 }
 
+// Rolling cache of a compressed layer.  Such a layer only ever attends to the first N_sink and
+// the last N_recent tokens (Eq. 2), so it stores nothing else: `sink_pages` pages hold positions
+// [0, 64 * sink_pages) for good, and `ring_pages` = ceil(N_recent / 64) + 1 further pages are
+// reused round-robin by all later 64-token blocks of the context.  A token at absolute position t
+// lives at this position of the request's (short) page table:
+__host__ __device__ __forceinline__ int32_t rolling_position(int32_t t, int32_t sink_pages, int32_t ring_pages)
+{
+    const int32_t block = t / kPage;
+    if (block < sink_pages) return t;
+    return (sink_pages + (block - sink_pages) % ring_pages) * kPage + t % kPage;
+}
+
 // The selection of one request: the caller's index list, or the index set of Eq. 2 of the
 // paper (attention sink + recent tokens) kept as two ranges, [0, ns) and [rs, M), so that no
 // index list has to exist in memory.  Position j of the selection is list[j] or, for ranges,
@@ -59,6 +72,7 @@ struct Selection {
     const int32_t *list;   // null for ranges
     int n;                 // selected tokens
     int ns, rs;            // ranges only: end of the sink range, start of the recent range
+    int sink_pages, ring_pages;   // ranges over a rolling cache (ring_pages > 0)
     bool bad;              // the length breaks the contract (n was set to 0)
 };
 
@@ -67,6 +81,8 @@ __device__ __forceinline__ Selection load_selection(const DecodeParams &p, int b
     Selection s;
     s.bad = false;
     s.ns = s.rs = 0;
+    s.sink_pages = p.sink_pages;
+    s.ring_pages = p.ring_pages;
     if (p.sel_idx != nullptr) {
         s.list = p.sel_idx + (size_t)b * p.max_sel;
         s.n = __ldg(p.sel_len + b);
@@ -77,7 +93,8 @@ __device__ __forceinline__ Selection load_selection(const DecodeParams &p, int b
     } else {
         s.list = nullptr;
         int m = __ldg(p.ctx_len + b);
-        if (m < 0 || (int64_t)m > (int64_t)p.max_pages * kPage) {
+        // a rolling cache holds contexts of any length in its few pages
+        if (m < 0 || (p.ring_pages == 0 && (int64_t)m > (int64_t)p.max_pages * kPage)) {
             s.bad = true;
             m = 0;
         }
@@ -93,7 +110,8 @@ __device__ __forceinline__ Selection load_selection(const DecodeParams &p, int b
 __device__ __forceinline__ int32_t selection_at(const Selection &s, int j)
 {
     if (s.list != nullptr) return __ldg(s.list + j);
-    return j < s.ns ? j : s.rs + (j - s.ns);
+    const int32_t t = j < s.ns ? j : s.rs + (j - s.ns);
+    return s.ring_pages > 0 ? rolling_position(t, s.sink_pages, s.ring_pages) : t;
 }
 
 // Logical token position -> physical pool row, or -1 if the entry breaks the index contract.

@@ -365,3 +365,37 @@ def test_sink_recent_attention_equals_dense_attention_over_a_cache_with_the_rest
                                                    np.arange(Ms, dtype=np.int32)[None],
                                                    np.array([Ms], np.int32), D_V, 0.2)
     assert np.array_equal(o_sparse, o_dense) and np.array_equal(l_sparse, l_dense)
+
+
+# ------------------------------------------------------------------ rolling cache layout
+
+def test_rolling_cache_keeps_every_token_of_the_index_set():
+    # Replaying the appends of a whole context and reading the index set back must return
+    # exactly the rows that were appended at those positions: no slot of the ring is reused
+    # while its token is still inside the recent window, whatever the context length.
+    from oracle import rolling, selection
+    rng = np.random.default_rng(90)
+    for n_sink, n_recent in ((64, 256), (5, 100), (0, 1), (70, 0), (130, 64), (1, 63)):
+        sink_pages, ring_pages = rolling.pages_per_request(n_sink, n_recent)
+        pages = sink_pages + ring_pages
+        table = rng.permutation(pages + 3)[:pages].astype(np.int32)         # scattered physical pages
+        for M in (0, 1, 63, 64, 65, 127, 128, 129, 500, 1000):
+            rows = rng.integers(1, 1 << 30, size=(M, 2)).astype(np.int64)   # two columns identify a token
+            pool = np.zeros((pages + 3, 64, 2), dtype=np.int64)
+            rolling.replay_appends(pool, table, rows, n_sink, n_recent)
+            want = selection.sink_recent(M, n_sink, n_recent)
+            got = rolling.selected_rows(table, M, n_sink, n_recent)
+            assert len(got) == len(want) and len(set(got.tolist())) == len(got)
+            assert np.array_equal(pool.reshape(-1, 2)[got], rows[want])
+
+
+def test_rolling_cache_sizes_and_fixed_points():
+    from oracle import rolling
+    assert rolling.pages_per_request(64, 2048) == (1, 33)
+    assert rolling.pages_per_request(0, 1) == (0, 2)
+    assert rolling.pages_per_request(65, 64) == (2, 2)
+    # the sink pages are never remapped; the first ring block follows them directly
+    for t in range(128):
+        assert rolling.position(t, 100, 64) == t
+    assert rolling.position(128, 100, 64) == 128 and rolling.position(128 + 64, 100, 64) == 192
+    assert rolling.position(128 + 2 * 64 + 5, 100, 64) == 128 + 5          # ring of 2 pages wraps
