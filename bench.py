@@ -155,11 +155,14 @@ def _oracle_sample(w, target_s=15.0, max_requests=None):
 WORKLOAD_HELP = ("config2 (default, the named benchmark) | config1 | config3 | config4 | "
                  "config5:<batch>:<selected>[:dense] (one sweep cell) | "
                  "eq2:<batch>:<n_sink>:<n_recent>[:list] (the paper's sink + recent rule on 32768-token contexts, "
-                 "through the range entry point, or with :list through the index-list entry point)")
+                 "through the range entry point, or with :list through the index-list entry point) | "
+                 "rolling:<batch>:<n_sink>:<n_recent> (the same rule over the rolling cache of a compressed layer, "
+                 "contexts of one million tokens)")
 
 
 def make_workload(spec, dev, batch):
     """Build a named workload and a one-line description of it."""
+    import numpy as np
     from paper_2511_22481_b200 import workloads as W
     if spec == "config2":
         w = W.config2_r1(dev, batch=batch)
@@ -185,6 +188,18 @@ def make_workload(spec, dev, batch):
         w.meta["entry"] = "list" if (len(f) > 4 and f[4] == "list") else "ranges"
         text = ("Eq. 2 selection: batch %s, 128 heads, ctx 32768, N_sink %s + N_recent %s, %s entry point, seed 30"
                 % (f[1], f[2], f[3], "index-list" if w.meta["entry"] == "list" else "range"))
+    elif spec.startswith("rolling:"):
+        from paper_2511_22481_b200 import binding as B
+        f = spec.split(":")
+        n_sink, n_recent = int(f[2]), int(f[3])
+        pages = B.omni_rolling_pages_per_request(n_sink, n_recent)
+        # the pool is the whole cache of the layer: pages per request x batch, shuffled; its contents stand
+        # for the sink and the last N_recent tokens of a context of one million tokens
+        w = W.sink_recent("rolling", 31, int(f[1]), 128, pages * 64, n_sink, n_recent, dev)
+        w.ctx_len = np.full(w.batch, 1000000, dtype=np.int64)
+        w.meta["entry"] = "rolling"
+        text = ("Eq. 2 selection over a rolling cache: batch %s, 128 heads, ctx 1000000, N_sink %d + N_recent %d, "
+                "%d pages per request, seed 31" % (f[1], n_sink, n_recent, pages))
     else:
         raise SystemExit("unknown --workload %r; choose %s" % (spec, WORKLOAD_HELP))
     return w, text
@@ -243,16 +258,17 @@ def main():
     flops = w.selected_tokens * w.heads * FLOP_PER_TOKEN_HEAD
     launches_per_step = B.omni_sparse_mla_num_launches(plan.desc)
 
-    ranges = w.meta.get("entry") == "ranges"
+    ranges = w.meta.get("entry") in ("ranges", "rolling")
+    range_entry = (B.omni_sparse_mla_decode_rolling if w.meta.get("entry") == "rolling"
+                   else B.omni_sparse_mla_decode_sink_recent)
     ctx_dev = torch.as_tensor(w.ctx_len, dtype=torch.int32).to(dev) if ranges else None
 
     def step(i, ev=None):
         if ev is not None:
             B.omni_sparse_mla_set_profile_events(ev[0], ev[1])
         if ranges:
-            B.omni_sparse_mla_decode_sink_recent(plan.desc, w.q, pools[i % clones], w.page_table, ctx_dev,
-                                                 w.meta["n_sink"], w.meta["n_recent"], plan.out, plan.lse,
-                                                 plan.workspace, plan.status)
+            range_entry(plan.desc, w.q, pools[i % clones], w.page_table, ctx_dev, w.meta["n_sink"],
+                        w.meta["n_recent"], plan.out, plan.lse, plan.workspace, plan.status)
         else:
             B.omni_sparse_mla_decode(plan.desc, w.q, pools[i % clones], w.page_table, w.sel_idx,
                                      w.sel_len, plan.out, plan.lse, plan.workspace, plan.status)

@@ -143,7 +143,9 @@ omni_status_t omni_sparse_mla_decode(const omni_mla_desc_t *desc, const void *q,
  * M = ctx_len[b] attends to [0, min(N_sink, M)) united with [max(M - N_recent, 0), M); where
  * the two ranges overlap the union is taken without repeats, so the selection is the whole
  * context once N_sink + N_recent >= M.  The result is that of omni_sparse_mla_decode on the
- * increasing list of those positions, bit for bit.
+ * increasing list of those positions (within rounding: the kernels walk the recent range in
+ * page-aligned tiles, which regroups the sums unless the range already starts on a page
+ * boundary right behind the sink; then the two results are bit-identical).
  *
  *   ctx_len    int32 [B], each in [0, max_pages_per_req * 64]; a value outside is treated like a
  *              bad sel_len (out = 0, lse = -inf, OMNI_DEV_BAD_INDEX)

@@ -66,12 +66,18 @@ __host__ __device__ __forceinline__ int32_t rolling_position(int32_t t, int32_t 
 
 // The selection of one request: the caller's index list, or the index set of Eq. 2 of the
 // paper (attention sink + recent tokens) kept as two ranges, [0, ns) and [rs, M), so that no
-// index list has to exist in memory.  Position j of the selection is list[j] or, for ranges,
-// j itself below ns and rs + (j - ns) from there on.
+// index list has to exist in memory.  Entry j of the selection is list[j] or, for ranges, j
+// itself below ns and a position of the recent range from `vstart` on.  Between the two ranges
+// up to 63 padding entries (kSelectionPad: "no token", weight zero, not an error) shift the
+// recent range so that position t sits at offset t mod 64 of its 64-entry tile: the tiles of the
+// recent window then coincide with pages and are loaded as boxes wherever the window starts,
+// instead of every tile straddling two pages.
+constexpr int32_t kSelectionPad = -2;
 struct Selection {
     const int32_t *list;   // null for ranges
-    int n;                 // selected tokens
+    int n;                 // entries (selected tokens, plus padding for ranges)
     int ns, rs;            // ranges only: end of the sink range, start of the recent range
+    int vstart;            // ranges only: entry of position rs
     int sink_pages, ring_pages;   // ranges over a rolling cache (ring_pages > 0)
     bool bad;              // the length breaks the contract (n was set to 0)
 };
@@ -80,7 +86,7 @@ __device__ __forceinline__ Selection load_selection(const DecodeParams &p, int b
 {
     Selection s;
     s.bad = false;
-    s.ns = s.rs = 0;
+    s.ns = s.rs = s.vstart = 0;
     s.sink_pages = p.sink_pages;
     s.ring_pages = p.ring_pages;
     if (p.sel_idx != nullptr) {
@@ -102,7 +108,8 @@ __device__ __forceinline__ Selection load_selection(const DecodeParams &p, int b
         // union without repeats
         s.ns = min(p.n_sink, m);
         s.rs = max(s.ns, m - min(p.n_recent, m));
-        s.n = s.ns + (m - s.rs);
+        s.vstart = s.ns + (m > s.rs ? ((s.rs - s.ns) % kPage) : 0);
+        s.n = s.vstart + (m - s.rs);
     }
     return s;
 }
@@ -110,7 +117,8 @@ __device__ __forceinline__ Selection load_selection(const DecodeParams &p, int b
 __device__ __forceinline__ int32_t selection_at(const Selection &s, int j)
 {
     if (s.list != nullptr) return __ldg(s.list + j);
-    const int32_t t = j < s.ns ? j : s.rs + (j - s.ns);
+    if (j >= s.ns && j < s.vstart) return kSelectionPad;
+    const int32_t t = j < s.ns ? j : s.rs + (j - s.vstart);
     return s.ring_pages > 0 ? rolling_position(t, s.sink_pages, s.ring_pages) : t;
 }
 

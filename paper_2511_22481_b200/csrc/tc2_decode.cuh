@@ -502,7 +502,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
                           bool &contig_lo, bool &contig_hi, bool &any_bad) {
         const int j0 = begin + tile * kC2Tile + lane, j1 = j0 + 32;
         const bool ok0 = x.pg0 >= 0 && (int64_t)x.pg0 < p.num_pages, ok1 = x.pg1 >= 0 && (int64_t)x.pg1 < p.num_pages;
-        any_bad |= (j0 < end && !ok0) || (j1 < end && !ok1);
+        any_bad |= (j0 < end && !ok0 && x.t0 != kSelectionPad) || (j1 < end && !ok1 && x.t1 != kSelectionPad);
         const int r0 = ok0 ? x.pg0 * kPage + x.t0 % kPage : -1, r1 = ok1 ? x.pg1 * kPage + x.t1 % kPage : -1;
         const uint32_t m0 = __ballot_sync(0xffffffffu, r0 >= 0), m1 = __ballot_sync(0xffffffffu, r1 >= 0);
         mask = (uint64_t)m0 | ((uint64_t)m1 << 32);

@@ -393,11 +393,11 @@ tc_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constan
             int64_t r0 = -1, r1 = -1;
             if (j0 < end) {
                 r0 = resolve_row(pt, t0, p.max_pages, p.num_pages);
-                any_bad |= (r0 < 0);
+                any_bad |= (r0 < 0 && t0 != kSelectionPad);
             }
             if (j1 < end) {
                 r1 = resolve_row(pt, t1, p.max_pages, p.num_pages);
-                any_bad |= (r1 < 0);
+                any_bad |= (r1 < 0 && t1 != kSelectionPad);
             }
             const uint32_t m0 = __ballot_sync(0xffffffffu, r0 >= 0), m1 = __ballot_sync(0xffffffffu, r1 >= 0);
             mask = (uint64_t)m0 | ((uint64_t)m1 << 32);

@@ -225,13 +225,29 @@ def test_sink_recent_ranges_match_oracle_on_the_index_set(flags, n_sink, n_recen
 
 
 def test_sink_recent_ranges_equal_the_list_path_bit_for_bit(flags):
-    ctx_tokens = [4096, 777, 130, 2048]
+    # recent ranges that start on a page boundary right behind a page-aligned sink: the range path
+    # walks exactly the tiles of the list path
+    ctx_tokens = [4096, 832, 130, 2048]
     w, ctx = _sink_recent_case(ctx_tokens, 64, 512, seed=61)
     for splits in (1, 2):
         plan = run_gpu(w, flags, num_splits=splits)
         out, lse, status = _run_ranges(w, ctx, 64, 512, flags, splits)
         assert status == 0
         assert torch.equal(out, plan.out) and torch.equal(lse, plan.lse)
+
+
+def test_sink_recent_ranges_on_unaligned_windows_stay_close_to_the_list_path(flags):
+    # any other start: the range path pads the recent range to page-aligned tiles, so sums are
+    # regrouped; both results are within the parity tolerance of the oracle, hence of each other
+    ctx_tokens = [4133, 777, 1001, 2049]
+    w, ctx = _sink_recent_case(ctx_tokens, 64, 512, seed=63)
+    ref_out, ref_lse, _ = oracle_subset(w)
+    for splits in (1, 2):
+        out, lse, status = _run_ranges(w, ctx, 64, 512, flags, splits)
+        assert status == 0
+        compare(out.cpu(), lse.cpu(), ref_out, ref_lse, "unaligned ranges S=%d" % splits)
+        plan = run_gpu(w, flags, num_splits=splits)
+        assert (out.float() - plan.out.float()).abs().max().item() <= 2e-3
 
 
 def test_sink_recent_bad_context_length_is_flagged():
