@@ -198,6 +198,25 @@ omni_status_t omni_sparse_mla_decode_rolling(const omni_mla_desc_t *desc, const 
                                              size_t workspace_bytes, int32_t *device_status, void *stream);
 
 /*
+ * Selection producer for token-level sparsity (the step before the decode call when the index
+ * set is "the k highest-scoring tokens", as in a top-k sparse attention variant; the paper
+ * itself only uses the sink + recent rule of Eq. 2).  For every request b with M = ctx_len[b]
+ * (clamped to [0, stride]) it writes into sel_idx[b] the positions of the min(k, M) largest of
+ * scores[b][0..M), in increasing order of position, and min(k, M) into sel_len[b]: exactly what
+ * omni_sparse_mla_decode reads (descriptor max_sel = k).  Scores compare as IEEE floats with
+ * -0 below +0 and NaN below everything; among equal scores at the threshold the lowest
+ * positions win, so the result is a deterministic function of the input.
+ *
+ *   scores   fp32 [batch, stride], stride <= 131072 (else OMNI_ERR_SHAPE)
+ *   ctx_len  int32 [batch]
+ *   k        1 <= k <= stride
+ *   sel_idx  int32 [batch, k] (written; entries at and beyond sel_len[b] are left untouched)
+ *   sel_len  int32 [batch]    (written)
+ */
+omni_status_t omni_topk_select(const float *scores, const int32_t *ctx_len, int32_t batch, int32_t stride,
+                               int32_t k, int32_t *sel_idx, int32_t *sel_len, void *stream);
+
+/*
  * Merge of split-KV partial results (the step that follows a partition of M into disjoint
  * ranges; Eq. 1 is recovered exactly because softmax normalisers add):
  *     lse[b,h]   = ln sum_s exp(part_lse[b,s,h])

@@ -28,6 +28,7 @@ EXPORTS = (
     "omni_version", "omni_status_string", "omni_sparse_mla_num_splits", "omni_sparse_mla_num_launches",
     "omni_sparse_mla_workspace_bytes", "omni_sparse_mla_decode", "omni_sparse_mla_decode_sink_recent",
     "omni_rolling_pages_per_request", "omni_kv_append_rolling", "omni_sparse_mla_decode_rolling",
+    "omni_topk_select",
     "omni_sparse_mla_combine",
     "omni_sparse_mla_validate", "omni_sparse_mla_resolve_rows",
     "omni_sparse_mla_host_staging_bytes", "omni_sparse_mla_decode_host",
@@ -89,6 +90,8 @@ def load() -> ctypes.CDLL:
     lib.omni_sparse_mla_decode_rolling.argtypes = [dp, vp, vp, vp, vp, i32, i32, vp, vp, vp, sz, vp, vp]
     lib.omni_kv_append_rolling.restype = ctypes.c_int
     lib.omni_kv_append_rolling.argtypes = [dp, vp, vp, vp, vp, i32, i32, vp, vp]
+    lib.omni_topk_select.restype = ctypes.c_int
+    lib.omni_topk_select.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp]
     lib.omni_rolling_pages_per_request.restype = i32
     lib.omni_rolling_pages_per_request.argtypes = [i32, i32]
     lib.omni_sparse_mla_combine.restype = ctypes.c_int
@@ -197,6 +200,16 @@ def omni_sparse_mla_decode_sink_recent(desc, q, kv_cache, page_table, ctx_len, n
         None if workspace is None else ctypes.c_void_p(workspace.data_ptr()), ws_bytes,
         _ptr(device_status, torch.int32, "cuda", "device_status"), _stream(stream))
     _check(code, "omni_sparse_mla_decode_sink_recent")
+
+
+def omni_topk_select(scores, ctx_len, k, sel_idx, sel_len, stream=None) -> None:
+    """Positions of the k largest scores of every request, as sel_idx / sel_len for the decode call."""
+    batch, stride = scores.shape
+    code = load().omni_topk_select(
+        _ptr(scores, torch.float32, "cuda", "scores"), _ptr(ctx_len, torch.int32, "cuda", "ctx_len"),
+        int(batch), int(stride), int(k), _ptr(sel_idx, torch.int32, "cuda", "sel_idx"),
+        _ptr(sel_len, torch.int32, "cuda", "sel_len"), _stream(stream))
+    _check(code, "omni_topk_select")
 
 
 def omni_rolling_pages_per_request(n_sink: int, n_recent: int) -> int:

@@ -9,6 +9,7 @@
 #include "simt_decode.cuh"
 #include "tc_decode.cuh"
 #include "tc2_decode.cuh"
+#include "topk_select.cuh"
 
 namespace omni {
 namespace {
@@ -368,6 +369,18 @@ omni_status_t omni_sparse_mla_decode_rolling(const omni_mla_desc_t *desc, const 
 {
     return decode_impl(desc, q, kv_cache, page_table, nullptr, nullptr, ctx_len, n_sink, n_recent, true, out, lse,
                        workspace, workspace_bytes, device_status, stream);
+}
+
+omni_status_t omni_topk_select(const float *scores, const int32_t *ctx_len, int32_t batch, int32_t stride,
+                               int32_t k, int32_t *sel_idx, int32_t *sel_len, void *stream)
+{
+    if (!scores || !ctx_len || !sel_idx || !sel_len) return OMNI_ERR_NULL;
+    if (batch < 1 || stride < 1 || stride > kTopkMaxContext || k < 1 || k > stride) return OMNI_ERR_SHAPE;
+    if (!aligned(scores, 4) || !aligned(ctx_len, 4) || !aligned(sel_idx, 4) || !aligned(sel_len, 4)) return OMNI_ERR_ALIGN;
+    const DeviceInfo &dev = device_info();
+    if (!dev.ok) return OMNI_ERR_CUDA;
+    if (dev.cc_major != 10) return OMNI_ERR_ARCH;
+    return launch_topk_select(scores, ctx_len, batch, stride, k, sel_idx, sel_len, static_cast<cudaStream_t>(stream));
 }
 
 int32_t omni_rolling_pages_per_request(int32_t n_sink, int32_t n_recent)
