@@ -157,7 +157,7 @@ WORKLOAD_HELP = ("config2 (default, the named benchmark) | config1 | config3 | c
                  "eq2:<batch>:<n_sink>:<n_recent>[:list] (the paper's sink + recent rule on 32768-token contexts, "
                  "through the range entry point, or with :list through the index-list entry point) | "
                  "rolling:<batch>:<n_sink>:<n_recent> (the same rule over the rolling cache of a compressed layer, "
-                 "contexts of one million tokens)")
+                 "contexts of one million tokens) | topk_select:<batch>:<ctx>:<k> (the top-k selection producer alone)")
 
 
 def make_workload(spec, dev, batch):
@@ -205,6 +205,104 @@ def make_workload(spec, dev, batch):
     return w, text
 
 
+def topk_arm(args, spec):
+    """`--workload topk_select:<batch>:<ctx>:<k>`: the selection producer alone (one launch per
+    step), scores of standard-normal noise, one GPU.  Same JSON shape as the decode arm."""
+    import numpy as np
+    import torch
+    from paper_2511_22481_b200 import binding as B
+    from paper_2511_22481_b200 import build as builder
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    parts = spec.split(":")
+    batch, ctx, k = (int(parts[1]), int(parts[2]), int(parts[3])) if len(parts) == 4 else (16, 131072, 2048)
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    builder.build()
+    B.load()
+    score_bytes = batch * ctx * 4
+    clones = max(2, -(-3 * L2_BYTES // score_bytes))           # bytes between two uses of a copy: 3 x L2
+    gen = torch.Generator(device="cpu").manual_seed(3)
+    scores_h = [torch.randn(batch, ctx, generator=gen).pin_memory() for _ in range(min(clones, 4))]
+    scores = [scores_h[i % len(scores_h)].to(dev) for i in range(clones)]
+    ctx_len = torch.full((batch,), ctx, dtype=torch.int32, device=dev)
+    sel_idx = torch.zeros(batch, k, dtype=torch.int32, device=dev)
+    sel_len = torch.zeros(batch, dtype=torch.int32, device=dev)
+    algo_bytes = score_bytes + batch * 4 + batch * min(k, ctx) * 4 + batch * 4
+
+    def step(i):
+        B.omni_topk_select(scores[i % clones], ctx_len, k, sel_idx, sel_len)
+
+    for i in range(args.warmup):
+        step(i)
+    sampler = ClockSampler(0)
+    torch.cuda.synchronize()
+    sampler.start()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for i in range(args.steps):
+        step(args.warmup + i)
+    t1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = t0.elapsed_time(t1) / args.steps
+
+    idx_h = torch.empty(batch, k, dtype=torch.int32).pin_memory()
+    len_h = torch.empty(batch, dtype=torch.int32).pin_memory()
+    stage = torch.empty(batch, ctx, device=dev)
+
+    def e2e_step(i):
+        stage.copy_(scores_h[i % len(scores_h)], non_blocking=True)
+        B.omni_topk_select(stage, ctx_len, k, sel_idx, sel_len)
+        idx_h.copy_(sel_idx, non_blocking=True)
+        len_h.copy_(sel_len, non_blocking=True)
+
+    for i in range(args.warmup):
+        e2e_step(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e2e_steps = min(args.steps, 500)
+    e0.record()
+    for i in range(e2e_steps):
+        e2e_step(i)
+    e1.record()
+    torch.cuda.synchronize()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+
+    peaks = _peaks()
+    achieved = algo_bytes / (ms * 1e-3) / 1e9
+    line = {
+        "metric": "top-k selection producer: score bytes consumed per second", "value": round(achieved, 2), "unit": "GB/s",
+        "us_per_step": round(ms * 1e3, 3), "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": round(ms, 6), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "u32 keys of f32 scores", "data": "synthetic",
+        "config": {"workload": "topk_select: batch %d, %d scores per request (standard normal, seed 3), k=%d" % (batch, ctx, k),
+                   "l2": "cold: %d score copies rotated (%.0f MB per cycle vs %.0f MB L2)"
+                         % (clones, clones * score_bytes / 1e6, L2_BYTES / 1e6)},
+        "clocks": clocks,
+        "e2e": {"value": round(algo_bytes / (e2e_ms * 1e-3) / 1e9, 2), "unit": "GB/s", "us_per_step": round(e2e_ms * 1e3, 3),
+                "h2d_bytes_per_step": score_bytes, "d2h_bytes_per_step": batch * k * 4 + batch * 4},
+        "gpu_launches": args.steps,
+        "roofline": {"bound": "hbm", "achieved": round(achieved, 2), "peak": peaks["hbm"], "unit": "GB/s",
+                     "frac": round(achieved / peaks["hbm"], 4), "traffic": None, "peak_source": peaks["source"],
+                     "kernel": "topk_select_kernel", "kernel_us_mean": round(ms * 1e3, 3),
+                     "algorithmic_bytes_per_launch": algo_bytes},
+    }
+    if not args.no_cpu_baseline:
+        from oracle.topk import topk_batch
+        sc = scores_h[0].numpy()
+        n, t_begin = 0, time.perf_counter()
+        while time.perf_counter() - t_begin < 10.0:
+            topk_batch(sc, [ctx] * batch, k)
+            n += 1
+        secs = time.perf_counter() - t_begin
+        line["cpu_baseline"] = {"value": round(n * algo_bytes / secs / 1e9, 5), "unit": "GB/s", "cores": 1, "kind": "oracle",
+                                "sample": "oracle top-k (numpy lexsort) on the whole batch, %d passes in %.1f s" % (n, secs)}
+    print(json.dumps(line), flush=True)
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -228,6 +326,10 @@ def main():
         if rank != 0:
             return 0
         return reference_arm(args)
+    if args.workload.startswith("topk_select"):
+        if rank != 0:
+            return 0
+        return topk_arm(args, args.workload)
 
     import torch
     import torch.distributed as dist

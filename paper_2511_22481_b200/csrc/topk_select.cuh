@@ -1,11 +1,11 @@
 // Selection producer for token-level sparsity: the positions of the k largest scores of every
 // request, written as the sel_idx / sel_len arrays the decode kernels read.
 //
-// One cluster of eight CTAs per request.  Every CTA loads an eighth of the request's scores
+// One cluster of up to eight CTAs per request.  Every CTA loads its share of the request's scores
 // ONCE, as order-preserving 32-bit keys, into shared memory; everything after that works on
 // shared memory.  A most-significant-digit radix select (four passes of 8 bits) finds the key
 // T of the k-th largest score: per pass every CTA histograms the digit of its keys that still
-// match the prefix, the eight histograms are summed through distributed shared memory, and each
+// match the prefix, the cluster's histograms are summed through distributed shared memory, and each
 // CTA scans the 256 bins for the digit that holds the k-th largest.  Then every key above T is
 // selected, and of the keys equal to T the ones at the lowest positions, as many as are still
 // missing; positions are written in increasing order, so the output is a deterministic function
@@ -48,168 +48,241 @@ __device__ __forceinline__ void topk_cluster_sync()
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
-// Exclusive prefix sum of one value per thread over the block (512 threads); also returns the total.
-__device__ __forceinline__ int topk_block_scan(int v, int *warp_sums, int &total)
-{
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    int inc = v;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        const int o = __shfl_up_sync(0xffffffffu, inc, d);
-        if (lane >= d) inc += o;
-    }
-    __syncthreads();                                      // warp_sums may still be read from the last call
-    if (lane == 31) warp_sums[warp] = inc;
-    __syncthreads();
-    int base = 0, tot = 0;
-#pragma unroll
-    for (int w = 0; w < kTopkThreads / 32; ++w) {
-        const int s = warp_sums[w];
-        if (w < warp) base += s;
-        tot += s;
-    }
-    total = tot;
-    return base + inc - v;
-}
+constexpr int kTopkWarps = kTopkThreads / 32;
 
-__global__ void __launch_bounds__(kTopkThreads, 1)
+struct TopkShared {
+    uint32_t replicas[256 * 32];     // digit histogram, one copy per lane: entry (digit, lane) at digit * 32 + lane
+    uint32_t published[2][256];      // this CTA's histogram of the current pass, read by the whole cluster
+    uint32_t counts[2];              // keys above / equal to the threshold in this chunk
+    uint32_t prefix, need;
+    uint32_t warp_sums[kTopkWarps];
+    uint32_t warp_gt[kTopkWarps], warp_eq[kTopkWarps];
+};
+
+__global__ void __launch_bounds__(kTopkThreads, 2)
 topk_select_kernel(const float *__restrict__ scores, const int32_t *__restrict__ ctx_len, int stride, int k,
                    int32_t *__restrict__ sel_idx, int32_t *__restrict__ sel_len)
 {
-    extern __shared__ uint32_t keys[];                    // kTopkChunk keys of this CTA
-    __shared__ uint32_t hist[256];                         // this CTA's digit histogram (read by the whole cluster)
-    __shared__ uint32_t counts[2];                         // keys above / equal to the threshold in this chunk
-    __shared__ uint32_t sh_prefix, sh_need;
-    __shared__ int warp_sums[kTopkThreads / 32];
+    extern __shared__ __align__(16) unsigned char topk_smem[];
+    TopkShared &sh = *reinterpret_cast<TopkShared *>(topk_smem);
+    uint32_t *keys = reinterpret_cast<uint32_t *>(topk_smem + sizeof(TopkShared));     // kTopkChunk keys of this CTA
 
-    uint32_t crank;
+    uint32_t crank, nranks;
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(crank));
-    const int b = blockIdx.x / kTopkCluster;
+    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(nranks));
+    OMNI_SPAN(0);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int b = blockIdx.x / nranks;
     int m = __ldg(ctx_len + b);
     m = max(0, min(m, stride));
     const int want = min(k, m);
-    const int chunk = (m + kTopkCluster - 1) / kTopkCluster;
+    const int chunk = (m + (int)nranks - 1) / (int)nranks;
     const int start = min(m, (int)crank * chunk), len = min(m, start + chunk) - start;
     const float *src = scores + (size_t)b * stride + start;
-    for (int i = threadIdx.x; i < len; i += kTopkThreads) keys[i] = topk_key(__ldg(src + i));
+    {
+        // scalar head up to a 16-byte boundary, 16-byte loads for the body, scalar tail
+        const int head = min(len, (int)((4u - (uint32_t)((reinterpret_cast<uintptr_t>(src) >> 2) & 3u)) & 3u));
+        const int body = (len - head) >> 2;
+        const float4 *src4 = reinterpret_cast<const float4 *>(src + head);
+#pragma unroll 8
+        for (int j = threadIdx.x; j < body; j += kTopkThreads) {
+            const float4 v = __ldg(src4 + j);
+            uint32_t *d = keys + head + 4 * j;
+            d[0] = topk_key(v.x);
+            d[1] = topk_key(v.y);
+            d[2] = topk_key(v.z);
+            d[3] = topk_key(v.w);
+        }
+        if ((int)threadIdx.x < head) keys[threadIdx.x] = topk_key(__ldg(src + threadIdx.x));
+        const int tail = head + 4 * body;
+        if (tail + (int)threadIdx.x < len) keys[tail + threadIdx.x] = topk_key(__ldg(src + tail + threadIdx.x));
+    }
+    for (int i = threadIdx.x; i < 256 * 32; i += kTopkThreads) sh.replicas[i] = 0;
 
     uint32_t prefix = 0, mask = 0, need = (uint32_t)want;
-    for (int shift = 24; shift >= 0; shift -= 8) {
-        if (threadIdx.x < 256) hist[threadIdx.x] = 0;
-        __syncthreads();
+    int pass = 0;
+    for (int shift = 24; shift >= 0; shift -= 8, ++pass) {
+        __syncthreads();                                   // keys stored (first pass), histogram copies zeroed
+        if (pass == 0) OMNI_SPAN(1);
+        // every lane adds into its own copy of the histogram: no two lanes of a warp ever meet on a
+        // word or a bank, however the digits are distributed
+#pragma unroll 8
         for (int i = threadIdx.x; i < len; i += kTopkThreads) {
             const uint32_t key = keys[i];
-            if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+            if ((key & mask) == prefix) atomicAdd(&sh.replicas[((key >> shift) & 255u) * 32 + lane], 1u);
         }
         __syncthreads();
-        topk_cluster_sync();                               // every CTA's histogram is complete and visible
-        if (threadIdx.x < 32) {
-            // lane l owns bins 8l .. 8l+7 of the summed histogram; find the bin of the need-th largest
-            uint32_t bins[8], mine = 0;
+        if (pass == 0) OMNI_SPAN(2);
+        {
+            // thread t sums half of the 32 copies of bin t / 2 (rotated start keeps the banks apart)
+            const int bin = threadIdx.x >> 1, half = threadIdx.x & 1;
+            uint32_t c = 0;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                uint32_t c = 0;
-                for (uint32_t r = 0; r < kTopkCluster; ++r) c += ld_cluster_u32(topk_map(&hist[8 * threadIdx.x + j], r));
-                bins[j] = c;
-                mine += c;
-            }
-            // above = keys in bins of higher lanes
-            uint32_t above = 0;
-            for (int l = 31; l >= 1; --l) {
-                const uint32_t other = __shfl_sync(0xffffffffu, mine, l);
-                if (l > (int)threadIdx.x) above += other;
-            }
-            const bool here = above < need && above + mine >= need;      // exactly one lane when need >= 1
-            if (here) {
-                uint32_t cum = above;
-                int digit = 8 * threadIdx.x;
+            for (int j = 0; j < 16; ++j) c += sh.replicas[bin * 32 + half * 16 + ((j + bin) & 15)];
+            c += __shfl_xor_sync(0xffffffffu, c, 1);
+            if (half == 0) sh.published[pass & 1][bin] = c;
+        }
+        __syncthreads();                                   // all copies read: they can be cleared for the next pass
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        for (int i = threadIdx.x; i < 256 * 32; i += kTopkThreads) sh.replicas[i] = 0;
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");      // every CTA's histogram is visible
+        if (pass == 0) OMNI_SPAN(3);
+        {
+            // threads 0..255: bin t of the histogram summed over the cluster, then the bin that holds
+            // the need-th largest key: keys in higher bins < need <= keys in this and higher bins
+            uint32_t c = 0;
+            if (threadIdx.x < 256)
+                for (uint32_t r = 0; r < nranks; ++r) c += ld_cluster_u32(topk_map(&sh.published[pass & 1][threadIdx.x], r));
+            uint32_t inc = c;                              // inclusive suffix sum within the warp
 #pragma unroll
-                for (int j = 7; j >= 0; --j) {
-                    if (cum + bins[j] >= need) {
-                        digit = 8 * threadIdx.x + j;
-                        break;
-                    }
-                    cum += bins[j];
-                }
-                sh_prefix = prefix | ((uint32_t)digit << shift);
-                sh_need = need - cum;
+            for (int d = 1; d < 32; d <<= 1) {
+                const uint32_t o = __shfl_down_sync(0xffffffffu, inc, d);
+                if (lane + d < 32) inc += o;
+            }
+            if (lane == 0) sh.warp_sums[warp] = inc;
+            __syncthreads();
+            uint32_t above = 0;                            // keys in the bins of higher warps
+            for (int w = warp + 1; w < 8; ++w) above += sh.warp_sums[w];
+            const uint32_t with_me = above + inc, higher = with_me - c;
+            if (threadIdx.x < 256 && higher < need && need <= with_me) {
+                sh.prefix = prefix | ((uint32_t)threadIdx.x << shift);
+                sh.need = need - higher;
             }
             if (need == 0 && threadIdx.x == 0) {
-                sh_prefix = prefix | (255u << shift);      // nothing to select: any threshold above all keys will do
-                sh_need = 0;
+                sh.prefix = prefix | (255u << shift);      // nothing to select: any threshold will do
+                sh.need = 0;
             }
         }
         __syncthreads();
-        prefix = sh_prefix;
-        need = sh_need;
+        prefix = sh.prefix;
+        need = sh.need;
         mask |= 255u << shift;
-        topk_cluster_sync();                               // all CTAs have read this pass's histograms
+        if (pass == 0) OMNI_SPAN(4);
+        // published[] alternates between passes, and the next pass's cluster barrier comes before
+        // anybody overwrites the copy read here
     }
-    // prefix is now the key T of the want-th largest score, need the number of keys equal to T still to take
+    // prefix is now the key T of the want-th largest score, need the number of keys equal to T still to take.
+    // Warp w owns the contiguous keys [w * per_warp, (w + 1) * per_warp) of the chunk.
     const uint32_t T = prefix;
+    OMNI_SPAN(5);
+    const int per_warp = ((len + kTopkWarps - 1) / kTopkWarps + 127) & ~127;
+    const int w_begin = min(len, warp * per_warp), w_end = min(len, w_begin + per_warp);
     uint32_t gt = 0, eq = 0;
-    for (int i = threadIdx.x; i < len; i += kTopkThreads) {
+#pragma unroll 8
+    for (int i = w_begin + lane; i < w_end; i += 32) {
         gt += keys[i] > T;
         eq += keys[i] == T;
     }
-    if (threadIdx.x < 2) counts[threadIdx.x] = 0;
-    __syncthreads();
-    if (want > 0) {
-        atomicAdd(&counts[0], gt);
-        atomicAdd(&counts[1], eq);
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+        gt += __shfl_xor_sync(0xffffffffu, gt, d);
+        eq += __shfl_xor_sync(0xffffffffu, eq, d);
+    }
+    if (lane == 0) {
+        sh.warp_gt[warp] = gt;
+        sh.warp_eq[warp] = eq;
     }
     __syncthreads();
+    uint32_t gt_before = 0, eq_before = 0, gt_all = 0, eq_all = 0;       // within this chunk, before this warp
+    for (int w = 0; w < kTopkWarps; ++w) {
+        const uint32_t g = sh.warp_gt[w], e = sh.warp_eq[w];
+        if (w < warp) {
+            gt_before += g;
+            eq_before += e;
+        }
+        gt_all += g;
+        eq_all += e;
+    }
+    if (threadIdx.x == 0) {
+        sh.counts[0] = gt_all;
+        sh.counts[1] = eq_all;
+    }
     topk_cluster_sync();
-    // selected entries and threshold ties in the chunks before this one
-    uint32_t out_base = 0, eq_before = 0;
+    OMNI_SPAN(6);
+    // threshold ties and keys above the threshold in the chunks before this one
     for (uint32_t r = 0; r < crank; ++r) {
-        const uint32_t g = ld_cluster_u32(topk_map(&counts[0], r)), e = ld_cluster_u32(topk_map(&counts[1], r));
-        const uint32_t take = eq_before < need ? min(e, need - eq_before) : 0u;
-        out_base += g + take;
-        eq_before += e;
+        gt_before += ld_cluster_u32(topk_map(&sh.counts[0], r));
+        eq_before += ld_cluster_u32(topk_map(&sh.counts[1], r));
     }
+    // entries written before this warp's first key: everything above T, and the first `need` ties
+    uint32_t run_eq = eq_before, run_out = gt_before + min(eq_before, need);
     int32_t *dst = sel_idx + (size_t)b * k;
-    int run_out = (int)out_base, run_eq = (int)eq_before;
-    for (int base = 0; base < len && want > 0; base += kTopkThreads) {
-        const int i = base + threadIdx.x;
-        const uint32_t key = i < len ? keys[i] : 0u;
-        const int is_eq = (i < len && key == T) ? 1 : 0;
-        int eq_total, sel_total;
-        const int eq_rank = run_eq + topk_block_scan(is_eq, warp_sums, eq_total);
-        const int sel = (i < len && (key > T || (is_eq && (uint32_t)eq_rank < need))) ? 1 : 0;
-        const int pos = run_out + topk_block_scan(sel, warp_sums, sel_total);
-        if (sel && pos < want) dst[pos] = start + i;
-        run_eq += eq_total;
-        run_out += sel_total;
+    const uint32_t lanes_below = (1u << lane) - 1u;
+    for (int base = w_begin; base < w_end && want > 0; base += 128) {
+        uint32_t key[4];
+        bool at_least[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int i = base + 32 * j + lane;
+            key[j] = i < w_end ? keys[i] : 0u;
+            at_least[j] = i < w_end && key[j] >= T;
+        }
+        if (!__any_sync(0xffffffffu, at_least[0] || at_least[1] || at_least[2] || at_least[3])) continue;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const bool is_eq = at_least[j] && key[j] == T;
+            const uint32_t eq_ballot = __ballot_sync(0xffffffffu, is_eq);
+            const uint32_t eq_rank = run_eq + __popc(eq_ballot & lanes_below);
+            const bool sel = at_least[j] && (!is_eq || eq_rank < need);
+            const uint32_t sel_ballot = __ballot_sync(0xffffffffu, sel);
+            const uint32_t pos = run_out + __popc(sel_ballot & lanes_below);
+            if (sel && pos < (uint32_t)want) dst[pos] = start + base + 32 * j + lane;
+            run_eq += __popc(eq_ballot);
+            run_out += __popc(sel_ballot);
+        }
     }
     if (crank == 0 && threadIdx.x == 0) sel_len[b] = want;
     topk_cluster_sync();                                   // nobody leaves while its counts may still be read
+    OMNI_SPAN(7);
+}
+
+// Cluster width for a launch: wide enough to hold `stride` keys, then wider while the grid still
+// fits the SMs in one wave.
+inline int topk_cluster_width(int batch, int stride, int sm_count)
+{
+    int width = 1;
+    while (width * kTopkChunk < stride) width *= 2;
+    while (width < kTopkCluster && (long long)batch * width * 2 <= sm_count) width *= 2;
+    return width;
 }
 
 inline omni_status_t launch_topk_select(const float *scores, const int32_t *ctx_len, int batch, int stride, int k,
-                                        int32_t *sel_idx, int32_t *sel_len, cudaStream_t stream)
+                                        int32_t *sel_idx, int32_t *sel_len, int sm_count, cudaStream_t stream)
 {
-    const size_t smem = (size_t)kTopkChunk * sizeof(uint32_t);
+    const size_t smem_need = sizeof(TopkShared) + (size_t)kTopkChunk * sizeof(uint32_t);
+    const size_t smem_alone = 120 * 1024;     // more than half an SM's shared memory: one CTA per SM
+    const int width = topk_cluster_width(batch, stride, sm_count);
     static bool attr_set[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return OMNI_ERR_CUDA;
     if (!attr_set[dev]) {
-        if (cudaFuncSetAttribute(topk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        if (cudaFuncSetAttribute(topk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_alone) != cudaSuccess)
             return OMNI_ERR_CUDA;
         attr_set[dev] = true;
     }
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(batch * kTopkCluster));
+    cfg.gridDim = dim3((unsigned)(batch * width));
     cfg.blockDim = dim3(kTopkThreads);
-    cfg.dynamicSmemBytes = smem;
+    cfg.dynamicSmemBytes = smem_alone;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = kTopkCluster;
+    attr[0].val.clusterDim.x = (unsigned)width;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    // A grid whose clusters are all resident with one CTA per SM spreads out instead of sharing SMs
+    // two by two; how many clusters of a width fit that way is asked once per device and width.
+    static int alone_clusters[64][4] = {};
+    int wlog = 0;
+    while ((1 << wlog) < width) ++wlog;
+    if (alone_clusters[dev][wlog] == 0) {
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, topk_select_kernel, &cfg) != cudaSuccess) n = -1;
+        alone_clusters[dev][wlog] = n > 0 ? n : -1;
+    }
+    if (batch > alone_clusters[dev][wlog]) cfg.dynamicSmemBytes = smem_need;
     return cudaLaunchKernelEx(&cfg, topk_select_kernel, scores, ctx_len, stride, k, sel_idx, sel_len) == cudaSuccess
                ? OMNI_OK
                : OMNI_ERR_CUDA;

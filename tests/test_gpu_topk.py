@@ -43,6 +43,16 @@ def test_random_scores_ragged_lengths(stride, k):
     _check(scores, ctx, k)
 
 
+@pytest.mark.parametrize("batch,stride,k", [(200, 5000, 300), (80, 20000, 1000), (40, 40000, 64), (1, 131072, 2048)])
+def test_cluster_widths_follow_batch_and_context(batch, stride, k):
+    """The launch picks 1, 2, 4 or 8 CTAs per request from the batch and the context length."""
+    rng = np.random.default_rng(batch)
+    scores = np.round(rng.standard_normal((batch, stride)) * 50).astype(np.float32)
+    ctx = rng.integers(0, stride + 1, batch).tolist()
+    ctx[0] = stride
+    _check(scores, ctx, k)
+
+
 @pytest.mark.parametrize("levels", [1, 2, 6, 300])
 def test_heavy_ties(levels):
     rng = np.random.default_rng(levels)
