@@ -65,7 +65,7 @@ topk_select_kernel(const float *__restrict__ scores, const int32_t *__restrict__
 {
     extern __shared__ __align__(16) unsigned char topk_smem[];
     TopkShared &sh = *reinterpret_cast<TopkShared *>(topk_smem);
-    uint32_t *keys = reinterpret_cast<uint32_t *>(topk_smem + sizeof(TopkShared));     // kTopkChunk keys of this CTA
+    uint32_t *keys = reinterpret_cast<uint32_t *>(topk_smem + sizeof(TopkShared));     // kTopkChunk keys of this CTA (+ 4 of slack)
 
     uint32_t crank, nranks;
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(crank));
@@ -81,17 +81,18 @@ topk_select_kernel(const float *__restrict__ scores, const int32_t *__restrict__
     const float *src = scores + (size_t)b * stride + start;
     {
         // scalar head up to a 16-byte boundary, 16-byte loads for the body, scalar tail
-        const int head = min(len, (int)((4u - (uint32_t)((reinterpret_cast<uintptr_t>(src) >> 2) & 3u)) & 3u));
+        // the keys sit in shared memory at the same offset from a 16-byte boundary as the scores in global
+        // memory, so that the body is stored with 16-byte stores too
+        const uint32_t misalign = (uint32_t)((reinterpret_cast<uintptr_t>(src) >> 2) & 3u);
+        keys += misalign;
+        const int head = min(len, (int)((4u - misalign) & 3u));
         const int body = (len - head) >> 2;
         const float4 *src4 = reinterpret_cast<const float4 *>(src + head);
 #pragma unroll 8
         for (int j = threadIdx.x; j < body; j += kTopkThreads) {
             const float4 v = __ldg(src4 + j);
-            uint32_t *d = keys + head + 4 * j;
-            d[0] = topk_key(v.x);
-            d[1] = topk_key(v.y);
-            d[2] = topk_key(v.z);
-            d[3] = topk_key(v.w);
+            *reinterpret_cast<uint4 *>(keys + head + 4 * j) =
+                make_uint4(topk_key(v.x), topk_key(v.y), topk_key(v.z), topk_key(v.w));
         }
         if ((int)threadIdx.x < head) keys[threadIdx.x] = topk_key(__ldg(src + threadIdx.x));
         const int tail = head + 4 * body;
@@ -131,8 +132,14 @@ topk_select_kernel(const float *__restrict__ scores, const int32_t *__restrict__
             // threads 0..255: bin t of the histogram summed over the cluster, then the bin that holds
             // the need-th largest key: keys in higher bins < need <= keys in this and higher bins
             uint32_t c = 0;
-            if (threadIdx.x < 256)
-                for (uint32_t r = 0; r < nranks; ++r) c += ld_cluster_u32(topk_map(&sh.published[pass & 1][threadIdx.x], r));
+            if (threadIdx.x < 256) {
+                uint32_t part[kTopkCluster];               // all remote loads in flight before the first use
+#pragma unroll
+                for (uint32_t r = 0; r < kTopkCluster; ++r)
+                    part[r] = r < nranks ? ld_cluster_u32(topk_map(&sh.published[pass & 1][threadIdx.x], r)) : 0u;
+#pragma unroll
+                for (uint32_t r = 0; r < kTopkCluster; ++r) c += part[r];
+            }
             uint32_t inc = c;                              // inclusive suffix sum within the warp
 #pragma unroll
             for (int d = 1; d < 32; d <<= 1) {
@@ -200,9 +207,18 @@ topk_select_kernel(const float *__restrict__ scores, const int32_t *__restrict__
     topk_cluster_sync();
     OMNI_SPAN(6);
     // threshold ties and keys above the threshold in the chunks before this one
-    for (uint32_t r = 0; r < crank; ++r) {
-        gt_before += ld_cluster_u32(topk_map(&sh.counts[0], r));
-        eq_before += ld_cluster_u32(topk_map(&sh.counts[1], r));
+    {
+        uint32_t g[kTopkCluster], e[kTopkCluster];         // all remote loads in flight before the first use
+#pragma unroll
+        for (uint32_t r = 0; r < kTopkCluster; ++r) {
+            g[r] = r < crank ? ld_cluster_u32(topk_map(&sh.counts[0], r)) : 0u;
+            e[r] = r < crank ? ld_cluster_u32(topk_map(&sh.counts[1], r)) : 0u;
+        }
+#pragma unroll
+        for (uint32_t r = 0; r < kTopkCluster; ++r) {
+            gt_before += g[r];
+            eq_before += e[r];
+        }
     }
     // entries written before this warp's first key: everything above T, and the first `need` ties
     uint32_t run_eq = eq_before, run_out = gt_before + min(eq_before, need);
@@ -249,7 +265,7 @@ inline int topk_cluster_width(int batch, int stride, int sm_count)
 inline omni_status_t launch_topk_select(const float *scores, const int32_t *ctx_len, int batch, int stride, int k,
                                         int32_t *sel_idx, int32_t *sel_len, int sm_count, cudaStream_t stream)
 {
-    const size_t smem_need = sizeof(TopkShared) + (size_t)kTopkChunk * sizeof(uint32_t);
+    const size_t smem_need = sizeof(TopkShared) + (size_t)(kTopkChunk + 4) * sizeof(uint32_t);
     const size_t smem_alone = 120 * 1024;     // more than half an SM's shared memory: one CTA per SM
     const int width = topk_cluster_width(batch, stride, sm_count);
     static bool attr_set[64] = {};
