@@ -510,11 +510,43 @@ def main():
     return 0
 
 
+def reference_topk_arm(args):
+    """The top-k oracle timed on one host core; each step is the whole batch of the workload."""
+    import torch
+    from oracle.topk import topk_batch
+    parts = args.workload.split(":")
+    batch, ctx, k = (int(parts[1]), int(parts[2]), int(parts[3])) if len(parts) == 4 else (16, 131072, 2048)
+    scores = torch.randn(batch, ctx, generator=torch.Generator().manual_seed(3)).numpy()
+    algo_bytes = batch * ctx * 4 + batch * 4 + batch * min(k, ctx) * 4 + batch * 4
+    steps = max(1, min(args.steps, 50))
+    for _ in range(min(args.warmup, 3)):
+        topk_batch(scores, [ctx] * batch, k)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        topk_batch(scores, [ctx] * batch, k)
+    secs = time.perf_counter() - t0
+    value = steps * algo_bytes / secs / 1e9
+    line = {
+        "impl": "reference", "metric": "top-k selection producer: score bytes consumed per second",
+        "value": round(value, 5), "unit": "GB/s", "n_gpus": args.gpus, "steps": steps, "warmup": min(args.warmup, 3),
+        "ms_per_step": round(secs / steps * 1e3, 3), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32 scores", "data": "synthetic",
+        "config": {"workload": "topk_select: batch %d, %d scores per request (standard normal, seed 3), k=%d" % (batch, ctx, k)},
+        "cpu_baseline": {"value": round(value, 5), "unit": "GB/s", "cores": 1, "kind": "oracle",
+                         "sample": "oracle top-k (numpy lexsort) on the whole batch, %d steps (capped at 50)" % steps},
+        "e2e": {"value": round(value, 5), "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+    return 0
+
+
 def reference_arm(args):
     """The oracle as the reference implementation, timed on host cores on a bounded sample."""
     import torch
     from paper_2511_22481_b200 import workloads as W
 
+    if args.workload.startswith("topk_select"):
+        return reference_topk_arm(args)
     # inputs of the same workload; a reduced pool is enough because only selected rows are read
     dev = "cuda" if torch.cuda.is_available() else "cpu"
     w, _ = make_workload(args.workload, dev, args.batch)
