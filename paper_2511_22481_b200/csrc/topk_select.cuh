@@ -19,6 +19,7 @@ namespace omni {
 constexpr int kTopkCluster = 8;
 constexpr int kTopkThreads = 512;
 constexpr int kTopkChunk = 16384;                        // keys per CTA held in shared memory
+constexpr int kTopkFew = 4096;                           // candidates below which a pass skips the lane-private copies
 constexpr int kTopkMaxContext = kTopkCluster * kTopkChunk;   // 131072 positions per request
 
 // float bits -> unsigned key with the same order; NaN sorts below everything
@@ -50,14 +51,16 @@ __device__ __forceinline__ void topk_cluster_sync()
 
 constexpr int kTopkWarps = kTopkThreads / 32;
 
-struct TopkShared {
+struct alignas(16) TopkShared {
     uint32_t replicas[256 * 32];     // digit histogram, one copy per lane: entry (digit, lane) at digit * 32 + lane
     uint32_t published[2][256];      // this CTA's histogram of the current pass, read by the whole cluster
     uint32_t counts[2];              // keys above / equal to the threshold in this chunk
-    uint32_t prefix, need;
+    uint32_t prefix, need;           // result of a digit search: the extended prefix, keys still to take in its bin
+    uint32_t bin_count;              // ... and the keys of the whole cluster in that bin
     uint32_t warp_sums[kTopkWarps];
     uint32_t warp_gt[kTopkWarps], warp_eq[kTopkWarps];
 };
+static_assert(sizeof(TopkShared) % 16 == 0, "the keys behind the control block are stored with 16-byte stores");
 
 __global__ void __launch_bounds__(kTopkThreads, 2)
 topk_select_kernel(const float *__restrict__ scores, const int32_t *__restrict__ ctx_len, int stride, int k,
@@ -71,6 +74,9 @@ topk_select_kernel(const float *__restrict__ scores, const int32_t *__restrict__
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(crank));
     asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(nranks));
     OMNI_SPAN(0);
+    // launched with programmatic stream serialization: nothing of the previous kernel in the stream is
+    // read or overwritten before this returns
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int b = blockIdx.x / nranks;
     int m = __ldg(ctx_len + b);
@@ -101,32 +107,45 @@ topk_select_kernel(const float *__restrict__ scores, const int32_t *__restrict__
     for (int i = threadIdx.x; i < 256 * 32; i += kTopkThreads) sh.replicas[i] = 0;
 
     uint32_t prefix = 0, mask = 0, need = (uint32_t)want;
+    bool few = false;                                      // at most kTopkFew keys of the cluster still match the prefix
     int pass = 0;
     for (int shift = 24; shift >= 0; shift -= 8, ++pass) {
         __syncthreads();                                   // keys stored (first pass), histogram copies zeroed
         if (pass == 0) OMNI_SPAN(1);
-        // every lane adds into its own copy of the histogram: no two lanes of a warp ever meet on a
-        // word or a bank, however the digits are distributed
+        if (few) {
+            // few keys are left in the cluster: they go straight into the published histogram
+            if (threadIdx.x < 256) sh.published[pass & 1][threadIdx.x] = 0;
+            __syncthreads();
 #pragma unroll 8
-        for (int i = threadIdx.x; i < len; i += kTopkThreads) {
-            const uint32_t key = keys[i];
-            if ((key & mask) == prefix) atomicAdd(&sh.replicas[((key >> shift) & 255u) * 32 + lane], 1u);
-        }
-        __syncthreads();
-        if (pass == 0) OMNI_SPAN(2);
-        {
-            // thread t sums half of the 32 copies of bin t / 2 (rotated start keeps the banks apart)
-            const int bin = threadIdx.x >> 1, half = threadIdx.x & 1;
-            uint32_t c = 0;
+            for (int i = threadIdx.x; i < len; i += kTopkThreads) {
+                const uint32_t key = keys[i];
+                if ((key & mask) == prefix) atomicAdd(&sh.published[pass & 1][(key >> shift) & 255u], 1u);
+            }
+            topk_cluster_sync();
+        } else {
+            // every lane adds into its own copy of the histogram: no two lanes of a warp ever meet on a
+            // word or a bank, however the digits are distributed
+#pragma unroll 8
+            for (int i = threadIdx.x; i < len; i += kTopkThreads) {
+                const uint32_t key = keys[i];
+                if ((key & mask) == prefix) atomicAdd(&sh.replicas[((key >> shift) & 255u) * 32 + lane], 1u);
+            }
+            __syncthreads();
+            if (pass == 0) OMNI_SPAN(2);
+            {
+                // thread t sums half of the 32 copies of bin t / 2 (rotated start keeps the banks apart)
+                const int bin = threadIdx.x >> 1, half = threadIdx.x & 1;
+                uint32_t c = 0;
 #pragma unroll
-            for (int j = 0; j < 16; ++j) c += sh.replicas[bin * 32 + half * 16 + ((j + bin) & 15)];
-            c += __shfl_xor_sync(0xffffffffu, c, 1);
-            if (half == 0) sh.published[pass & 1][bin] = c;
+                for (int j = 0; j < 16; ++j) c += sh.replicas[bin * 32 + half * 16 + ((j + bin) & 15)];
+                c += __shfl_xor_sync(0xffffffffu, c, 1);
+                if (half == 0) sh.published[pass & 1][bin] = c;
+            }
+            __syncthreads();                                   // all copies read: they can be cleared for the next pass
+            asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+            for (int i = threadIdx.x; i < 256 * 32; i += kTopkThreads) sh.replicas[i] = 0;
+            asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");      // every CTA's histogram is visible
         }
-        __syncthreads();                                   // all copies read: they can be cleared for the next pass
-        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-        for (int i = threadIdx.x; i < 256 * 32; i += kTopkThreads) sh.replicas[i] = 0;
-        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");      // every CTA's histogram is visible
         if (pass == 0) OMNI_SPAN(3);
         {
             // threads 0..255: bin t of the histogram summed over the cluster, then the bin that holds
@@ -154,15 +173,18 @@ topk_select_kernel(const float *__restrict__ scores, const int32_t *__restrict__
             if (threadIdx.x < 256 && higher < need && need <= with_me) {
                 sh.prefix = prefix | ((uint32_t)threadIdx.x << shift);
                 sh.need = need - higher;
+                sh.bin_count = c;
             }
             if (need == 0 && threadIdx.x == 0) {
                 sh.prefix = prefix | (255u << shift);      // nothing to select: any threshold will do
                 sh.need = 0;
+                sh.bin_count = 0;
             }
         }
         __syncthreads();
         prefix = sh.prefix;
         need = sh.need;
+        few = sh.bin_count <= (uint32_t)kTopkFew;
         mask |= 255u << shift;
         if (pass == 0) OMNI_SPAN(4);
         // published[] alternates between passes, and the next pass's cluster barrier comes before
@@ -281,13 +303,15 @@ inline omni_status_t launch_topk_select(const float *scores, const int32_t *ctx_
     cfg.blockDim = dim3(kTopkThreads);
     cfg.dynamicSmemBytes = smem_alone;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = (unsigned)width;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     // A grid whose clusters are all resident with one CTA per SM spreads out instead of sharing SMs
     // two by two; how many clusters of a width fit that way is asked once per device and width.
     static int alone_clusters[64][4] = {};
