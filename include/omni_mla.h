@@ -262,8 +262,14 @@ omni_status_t omni_sparse_mla_resolve_rows(const omni_mla_desc_t *desc,
  *
  *   staging, staging_bytes   device scratch for the per-step tensors, at least
  *                            omni_sparse_mla_host_staging_bytes(desc), 256-byte aligned
- * The copies and kernels are all enqueued on `stream`; the host buffers may be read after the
- * stream is synchronised.
+ *                            (the size includes split-KV scratch for the two-part schedule below)
+ * Everything is ordered on `stream`: the host buffers may be read after the stream is
+ * synchronised.  From a batch of a few megabytes of q and out on (at least 4 requests), the
+ * call runs the batch as two parts: the second part's q copy and, later, its kernel and copies
+ * out go to a stream the library creates once per device, which waits for `stream` at the
+ * start and which `stream` waits for at the end, so that copies in, kernels and copies out of
+ * the two parts overlap (PCIe carries both directions at once).  `workspace` is used only when
+ * the batch runs as one part.
  */
 size_t omni_sparse_mla_host_staging_bytes(const omni_mla_desc_t *desc);
 omni_status_t omni_sparse_mla_decode_host(const omni_mla_desc_t *desc, const void *q_host,

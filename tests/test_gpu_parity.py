@@ -300,6 +300,27 @@ def test_host_buffer_entry_point(flags):
     compare(out_h, lse_h, ref_out, ref_lse, "host entry point")
 
 
+@pytest.mark.parametrize("batch", [8, 9])
+def test_host_buffer_entry_point_two_halves(flags, batch):
+    """From 8 requests of 128 heads on, the host entry point runs the batch as two halves on two
+    streams; the result must not depend on that."""
+    w = W.config4_topk(DEV, batch=batch, ctx_pages=32, k=300)
+    desc = B.make_desc(w.batch, w.heads, w.num_pages, w.max_pages_per_req, w.max_sel, w.scale, flags=flags)
+    staging = torch.empty(B.omni_sparse_mla_host_staging_bytes(desc), dtype=torch.uint8, device=DEV)
+    ws = torch.empty(max(1, B.omni_sparse_mla_workspace_bytes(desc)), dtype=torch.uint8, device=DEV)
+    pin = lambda t: t.cpu().pin_memory()
+    q, pt, si, sl = pin(w.q), pin(w.page_table), pin(w.sel_idx), pin(w.sel_len)
+    out_h = torch.full((w.batch, w.heads, 512), float("nan"), dtype=torch.bfloat16).pin_memory()
+    lse_h = torch.full((w.batch, w.heads), float("nan"), dtype=torch.float32).pin_memory()
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    for _ in range(3):                       # back-to-back calls reuse the staging buffer
+        B.omni_sparse_mla_decode_host(desc, q, w.kv_cache, pt, si, sl, out_h, lse_h, staging, ws, status)
+    torch.cuda.current_stream().synchronize()            # the caller's stream alone covers both halves
+    assert int(status.item()) == 0
+    ref_out, ref_lse, _ = oracle_subset(w)
+    compare(out_h, lse_h, ref_out, ref_lse, "host entry point, two halves")
+
+
 # ------------------------------------------------------------------ full benchmark sizes, sampled
 
 def test_config2_full_size_sampled(flags):
