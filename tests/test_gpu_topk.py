@@ -80,6 +80,17 @@ def test_keys_that_differ_only_in_low_bits():
     _check(bits.view(np.float32), [30000, 12345], 4096)
 
 
+@pytest.mark.parametrize("m", [4095, 4096, 4097, 9000])
+def test_candidate_counts_around_the_direct_histogram_threshold(m):
+    """Scores in [1, 2) share their first key digit, so exactly m keys stay candidates after the
+    first pass: on both sides of the count (4096) below which a pass adds straight into the
+    published histogram."""
+    rng = np.random.default_rng(m)
+    scores = (1.0 + rng.random((3, 9000))).astype(np.float32)
+    scores[1] = np.round(scores[1] * 64) / 64              # ties inside the shared digit
+    _check(scores, [m, m, m - 1], 1000)
+
+
 def test_argument_checks():
     s = torch.zeros(2, 16, device=DEV)
     cl = torch.zeros(2, dtype=torch.int32, device=DEV)
