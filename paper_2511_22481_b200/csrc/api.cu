@@ -380,7 +380,7 @@ omni_status_t omni_topk_select(const float *scores, const int32_t *ctx_len, int3
     const DeviceInfo &dev = device_info();
     if (!dev.ok) return OMNI_ERR_CUDA;
     if (dev.cc_major != 10) return OMNI_ERR_ARCH;
-    return launch_topk_select(scores, ctx_len, batch, stride, k, sel_idx, sel_len, dev.sm_count, static_cast<cudaStream_t>(stream));
+    return launch_topk_select(scores, ctx_len, batch, stride, k, sel_idx, sel_len, static_cast<cudaStream_t>(stream));
 }
 
 int32_t omni_rolling_pages_per_request(int32_t n_sink, int32_t n_recent)

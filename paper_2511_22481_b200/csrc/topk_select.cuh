@@ -18,9 +18,9 @@ namespace omni {
 
 constexpr int kTopkCluster = 8;
 constexpr int kTopkThreads = 512;
-constexpr int kTopkChunk = 16384;                        // keys per CTA held in shared memory
+constexpr int kTopkChunk = 24576;                        // most keys a CTA holds in shared memory (96 KiB)
 constexpr int kTopkFew = 4096;                           // candidates below which a pass skips the lane-private copies
-constexpr int kTopkMaxContext = kTopkCluster * kTopkChunk;   // 131072 positions per request
+constexpr int kTopkMaxContext = 131072;                  // positions per request
 
 // float bits -> unsigned key with the same order; NaN sorts below everything
 __device__ __forceinline__ uint32_t topk_key(float f)
@@ -68,7 +68,7 @@ topk_select_kernel(const float *__restrict__ scores, const int32_t *__restrict__
 {
     extern __shared__ __align__(16) unsigned char topk_smem[];
     TopkShared &sh = *reinterpret_cast<TopkShared *>(topk_smem);
-    uint32_t *keys = reinterpret_cast<uint32_t *>(topk_smem + sizeof(TopkShared));     // kTopkChunk keys of this CTA (+ 4 of slack)
+    uint32_t *keys = reinterpret_cast<uint32_t *>(topk_smem + sizeof(TopkShared));     // this CTA's keys: ceil(stride / cluster width) (+ 4 of slack)
 
     uint32_t crank, nranks;
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(crank));
@@ -82,7 +82,7 @@ topk_select_kernel(const float *__restrict__ scores, const int32_t *__restrict__
     int m = __ldg(ctx_len + b);
     m = max(0, min(m, stride));
     const int want = min(k, m);
-    const int chunk = (m + (int)nranks - 1) / (int)nranks;
+    const int chunk = ((m + (int)nranks - 1) / (int)nranks + 3) & ~3;      // a multiple of four keeps the 16-byte loads aligned
     const int start = min(m, (int)crank * chunk), len = min(m, start + chunk) - start;
     const float *src = scores + (size_t)b * stride + start;
     {
@@ -274,36 +274,28 @@ topk_select_kernel(const float *__restrict__ scores, const int32_t *__restrict__
     OMNI_SPAN(7);
 }
 
-// Cluster width for a launch: wide enough to hold `stride` keys, then wider while the grid still
-// fits the SMs in one wave.
-inline int topk_cluster_width(int batch, int stride, int sm_count)
-{
-    int width = 1;
-    while (width * kTopkChunk < stride) width *= 2;
-    while (width < kTopkCluster && (long long)batch * width * 2 <= sm_count) width *= 2;
-    return width;
-}
+// Launch shape.  A CTA costs about 4 us plus 0.4 us per CTA of its cluster, plus 0.6 us per 1024 keys
+// when it has its SM to itself and 0.85 us per 1024 keys when two CTAs share an SM (fitted to
+// measurements).  Every width from 1 to 8 that holds the context is priced with the number of clusters
+// of that width the device keeps resident, alone on their SMs or two to an SM, and the cheapest wins.
+struct TopkShape {
+    int width;
+    size_t smem;
+};
 
-inline omni_status_t launch_topk_select(const float *scores, const int32_t *ctx_len, int batch, int stride, int k,
-                                        int32_t *sel_idx, int32_t *sel_len, int sm_count, cudaStream_t stream)
+constexpr size_t kTopkSmemAlone = 120 * 1024;            // more than half an SM's shared memory: one CTA per SM
+constexpr size_t kTopkSmemPair = 112 * 1024;             // two CTAs of up to this much fit one SM
+
+inline size_t topk_smem_need(int chunk) { return sizeof(TopkShared) + (size_t)(chunk + 4) * sizeof(uint32_t); }
+
+inline void topk_launch_config(cudaLaunchConfig_t &cfg, cudaLaunchAttribute *attr, int batch, int width, size_t smem,
+                               cudaStream_t stream)
 {
-    const size_t smem_need = sizeof(TopkShared) + (size_t)(kTopkChunk + 4) * sizeof(uint32_t);
-    const size_t smem_alone = 120 * 1024;     // more than half an SM's shared memory: one CTA per SM
-    const int width = topk_cluster_width(batch, stride, sm_count);
-    static bool attr_set[64] = {};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return OMNI_ERR_CUDA;
-    if (!attr_set[dev]) {
-        if (cudaFuncSetAttribute(topk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_alone) != cudaSuccess)
-            return OMNI_ERR_CUDA;
-        attr_set[dev] = true;
-    }
-    cudaLaunchConfig_t cfg = {};
+    cfg = cudaLaunchConfig_t{};
     cfg.gridDim = dim3((unsigned)(batch * width));
     cfg.blockDim = dim3(kTopkThreads);
-    cfg.dynamicSmemBytes = smem_alone;
+    cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = (unsigned)width;
     attr[0].val.clusterDim.y = 1;
@@ -312,17 +304,69 @@ inline omni_status_t launch_topk_select(const float *scores, const int32_t *ctx_
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    // A grid whose clusters are all resident with one CTA per SM spreads out instead of sharing SMs
-    // two by two; how many clusters of a width fit that way is asked once per device and width.
-    static int alone_clusters[64][4] = {};
-    int wlog = 0;
-    while ((1 << wlog) < width) ++wlog;
-    if (alone_clusters[dev][wlog] == 0) {
+}
+
+// Clusters of `width` resident at once (asked once per device, width and mode; at least 1).
+inline int topk_resident_clusters(int dev, int width, bool alone)
+{
+    static int cache[64][kTopkCluster + 1][2] = {};
+    int &slot = cache[dev][width][alone ? 1 : 0];
+    if (slot == 0) {
+        cudaLaunchConfig_t cfg;
+        cudaLaunchAttribute attr[2];
+        topk_launch_config(cfg, attr, 1, width, alone ? kTopkSmemAlone : kTopkSmemPair, nullptr);
+        cfg.numAttrs = 1;                                  // the cluster shape is all the query needs
         int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, topk_select_kernel, &cfg) != cudaSuccess) n = -1;
-        alone_clusters[dev][wlog] = n > 0 ? n : -1;
+        if (cudaOccupancyMaxActiveClusters(&n, topk_select_kernel, &cfg) != cudaSuccess) n = 0;
+        slot = n > 0 ? n : 1;
     }
-    if (batch > alone_clusters[dev][wlog]) cfg.dynamicSmemBytes = smem_need;
+    return slot;
+}
+
+inline TopkShape topk_shape(int dev, int batch, int stride)
+{
+    TopkShape best = {kTopkCluster, topk_smem_need(kTopkChunk)};
+    double best_cost = 1e30;
+    for (int width = kTopkCluster; width >= 1; --width) {
+        const int chunk = ((stride + width - 1) / width + 3) & ~3;
+        if (chunk > kTopkChunk) break;                     // narrower clusters cannot hold the context
+        const size_t need = topk_smem_need(chunk);
+        const double per_key = chunk / 1024.0;
+        const int alone = topk_resident_clusters(dev, width, true);
+        const double fixed = 4.0 + 0.4 * width + ((width & (width - 1)) ? 0.5 : 0.0);   // odd widths measured slightly slower
+        const double cost_alone = ((batch + alone - 1) / alone) * (fixed + 0.6 * per_key);
+        if (cost_alone < best_cost) {
+            best_cost = cost_alone;
+            best = {width, need > kTopkSmemAlone ? need : kTopkSmemAlone};
+        }
+        if (need <= kTopkSmemPair) {
+            const int paired = topk_resident_clusters(dev, width, false);
+            const double cost_pair = ((batch + paired - 1) / paired) * (fixed + 0.85 * per_key);
+            if (cost_pair < best_cost) {
+                best_cost = cost_pair;
+                best = {width, need};
+            }
+        }
+    }
+    return best;
+}
+
+inline omni_status_t launch_topk_select(const float *scores, const int32_t *ctx_len, int batch, int stride, int k,
+                                        int32_t *sel_idx, int32_t *sel_len, cudaStream_t stream)
+{
+    static bool attr_set[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return OMNI_ERR_CUDA;
+    if (!attr_set[dev]) {
+        if (cudaFuncSetAttribute(topk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)topk_smem_need(kTopkChunk)) != cudaSuccess)
+            return OMNI_ERR_CUDA;
+        attr_set[dev] = true;
+    }
+    const TopkShape shape = topk_shape(dev, batch, stride);
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[2];
+    topk_launch_config(cfg, attr, batch, shape.width, shape.smem, stream);
     return cudaLaunchKernelEx(&cfg, topk_select_kernel, scores, ctx_len, stride, k, sel_idx, sel_len) == cudaSuccess
                ? OMNI_OK
                : OMNI_ERR_CUDA;
