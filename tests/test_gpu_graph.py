@@ -63,3 +63,46 @@ def test_layer_loop_in_one_cuda_graph_matches_eager():
         assert torch.equal(graph_out[l], eager_out[l]) and torch.equal(graph_lse[l], eager_lse[l]), l
     # the sparse and the dense layers do differ (the pattern is not ignored)
     assert not torch.equal(eager_out[0], eager_out[1])
+
+
+def test_topk_producer_and_decode_in_one_cuda_graph_match_eager():
+    """scores -> top-k kernel -> decode kernel captured as one graph; replays with new scores follow them."""
+    k, ctx_pages = 512, 40
+    w = W.config4_topk(DEV, batch=4, ctx_pages=ctx_pages, k=k)
+    ctx = ctx_pages * 64
+    g = torch.Generator(device=DEV).manual_seed(72)
+    scores = torch.randn(w.batch, ctx, generator=g, device=DEV)
+    ctx_len = torch.tensor([ctx, ctx - 7, 300, ctx], dtype=torch.int32, device=DEV)
+    desc = B.make_desc(w.batch, 128, w.num_pages, w.max_pages_per_req, k, w.scale)
+    ws = torch.empty(max(1, B.omni_sparse_mla_workspace_bytes(desc)), dtype=torch.uint8, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+
+    def chain(sel_idx, sel_len, out, lse):
+        B.omni_topk_select(scores, ctx_len, k, sel_idx, sel_len)
+        B.omni_sparse_mla_decode(desc, w.q, w.kv_cache, w.page_table, sel_idx, sel_len, out, lse, ws, status)
+
+    def buffers():
+        return (torch.zeros(w.batch, k, dtype=torch.int32, device=DEV), torch.zeros(w.batch, dtype=torch.int32, device=DEV),
+                torch.empty((w.batch, 128, 512), dtype=torch.bfloat16, device=DEV),
+                torch.empty((w.batch, 128), dtype=torch.float32, device=DEV))
+
+    eager = buffers()
+    chain(*eager)                                   # also the warm-up
+    torch.cuda.synchronize()
+    captured = buffers()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        chain(*captured)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for a, b in zip(captured, eager):
+        assert torch.equal(a, b)
+    # new scores in the same buffer: the replay selects and attends accordingly
+    scores.copy_(torch.randn(w.batch, ctx, generator=g, device=DEV))
+    chain(*eager)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for a, b in zip(captured, eager):
+        assert torch.equal(a, b)
