@@ -189,10 +189,12 @@ topk_select_kernel(const float *__restrict__ scores, const int32_t *__restrict__
         if (pass == 0) OMNI_SPAN(4);
         // published[] alternates between passes, and the next pass's cluster barrier comes before
         // anybody overwrites the copy read here
+        if (need == sh.bin_count) break;                   // every key left under the prefix is taken: the lower digits decide nothing
     }
-    // prefix is now the key T of the want-th largest score, need the number of keys equal to T still to take.
+    // Keys above the prefix's range are selected, keys inside it (all digits searched: keys equal to the
+    // threshold) tie for the `need` places left, lowest positions first.
     // Warp w owns the contiguous keys [w * per_warp, (w + 1) * per_warp) of the chunk.
-    const uint32_t T = prefix;
+    const uint32_t T = prefix | ~mask;                     // largest key under the prefix
     OMNI_SPAN(5);
     const int per_warp = ((len + kTopkWarps - 1) / kTopkWarps + 127) & ~127;
     const int w_begin = min(len, warp * per_warp), w_end = min(len, w_begin + per_warp);
@@ -200,7 +202,7 @@ topk_select_kernel(const float *__restrict__ scores, const int32_t *__restrict__
 #pragma unroll 8
     for (int i = w_begin + lane; i < w_end; i += 32) {
         gt += keys[i] > T;
-        eq += keys[i] == T;
+        eq += (keys[i] & mask) == prefix;
     }
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) {
@@ -253,12 +255,12 @@ topk_select_kernel(const float *__restrict__ scores, const int32_t *__restrict__
         for (int j = 0; j < 4; ++j) {
             const int i = base + 32 * j + lane;
             key[j] = i < w_end ? keys[i] : 0u;
-            at_least[j] = i < w_end && key[j] >= T;
+            at_least[j] = i < w_end && key[j] >= prefix;
         }
         if (!__any_sync(0xffffffffu, at_least[0] || at_least[1] || at_least[2] || at_least[3])) continue;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const bool is_eq = at_least[j] && key[j] == T;
+            const bool is_eq = at_least[j] && (key[j] & mask) == prefix;
             const uint32_t eq_ballot = __ballot_sync(0xffffffffu, is_eq);
             const uint32_t eq_rank = run_eq + __popc(eq_ballot & lanes_below);
             const bool sel = at_least[j] && (!is_eq || eq_rank < need);
