@@ -212,6 +212,11 @@ omni_status_t omni_sparse_mla_decode_rolling(const omni_mla_desc_t *desc, const 
  *   k        1 <= k <= stride
  *   sel_idx  int32 [batch, k] (written; entries at and beyond sel_len[b] are left untouched)
  *   sel_len  int32 [batch]    (written)
+ * All pointers are device pointers owned by the caller; nothing is allocated.  One kernel is
+ * enqueued on `stream` (NULL: the default stream) and the call returns without waiting for it.
+ * Errors: OMNI_ERR_NULL (a null pointer), OMNI_ERR_SHAPE (batch < 1, k outside [1, stride],
+ * stride outside [1, 131072]), OMNI_ERR_ALIGN (a pointer not 4-byte aligned), OMNI_ERR_ARCH
+ * (not an sm_100 device), OMNI_ERR_CUDA (the launch failed).
  */
 omni_status_t omni_topk_select(const float *scores, const int32_t *ctx_len, int32_t batch, int32_t stride,
                                int32_t k, int32_t *sel_idx, int32_t *sel_len, void *stream);
