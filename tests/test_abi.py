@@ -106,6 +106,21 @@ def test_sink_recent_entry_point_checks_its_arguments(lib):
     assert B.omni_sparse_mla_num_launches(_desc(batch=0)) == 0
 
 
+def test_topk_select_checks_its_arguments(lib):
+    ok = ctypes.c_void_p(4096)
+    i32 = ctypes.c_int32
+    call = lambda scores, ctx, batch, stride, k, idx, ln: lib.omni_topk_select(
+        scores, ctx, i32(batch), i32(stride), i32(k), idx, ln, None)
+    for missing in range(4):
+        ptrs = [ok] * 4
+        ptrs[missing] = None
+        assert call(ptrs[0], ptrs[1], 2, 64, 8, ptrs[2], ptrs[3]) == 1        # OMNI_ERR_NULL
+    for batch, stride, k in ((0, 64, 8), (2, 0, 1), (2, 64, 0), (2, 64, 65), (2, 131073, 8)):
+        assert call(ok, ok, batch, stride, k, ok, ok) == 2                    # OMNI_ERR_SHAPE
+    odd = ctypes.c_void_p(4096 + 2)
+    assert call(odd, ok, 2, 64, 8, ok, ok) == 3 and call(ok, ok, 2, 64, 8, odd, ok) == 3      # OMNI_ERR_ALIGN
+
+
 def test_workspace_grows_with_forced_splits(lib):
     a = B.omni_sparse_mla_workspace_bytes(_desc(num_splits=1))
     b = B.omni_sparse_mla_workspace_bytes(_desc(num_splits=4))
