@@ -12,6 +12,8 @@
 // of the scores (ties included).
 #pragma once
 
+#include <mutex>
+
 #include "common.cuh"
 
 namespace omni {
@@ -311,7 +313,9 @@ inline void topk_launch_config(cudaLaunchConfig_t &cfg, cudaLaunchAttribute *att
 // Clusters of `width` resident at once (asked once per device, width and mode; at least 1).
 inline int topk_resident_clusters(int dev, int width, bool alone)
 {
+    static std::mutex lock;                                // callers on several host threads share the table
     static int cache[64][kTopkCluster + 1][2] = {};
+    std::lock_guard<std::mutex> guard(lock);
     int &slot = cache[dev][width][alone ? 1 : 0];
     if (slot == 0) {
         cudaLaunchConfig_t cfg;
