@@ -11,7 +11,14 @@
  *
  * Conventions shared by every entry point
  *   - Unless a parameter says "host", pointers are DEVICE pointers owned by the caller.
- *     The library allocates no device memory and keeps no per-call state.
+ *     The library allocates no device memory and keeps no per-call state.  What it does keep,
+ *     per process: per-device facts looked up once (SM count, kernel attributes, how many
+ *     merging clusters fit), a table of tensor-map encodings keyed by (base address, sizes)
+ *     so that repeated calls on the same buffers skip the encoding, one side stream per
+ *     device for omni_sparse_mla_decode_host, the address of the static scratch array of
+ *     omni_sparse_mla_decode_static, and the two event handles of
+ *     omni_sparse_mla_set_profile_events.  All of it is guarded for use from several host
+ *     threads except the profile events.
  *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*).  Errors the host
  *     can see (null pointer, bad shape, misalignment, short workspace) are returned at once
  *     and nothing is launched.
@@ -29,7 +36,10 @@
 #include <stdint.h>
 
 #ifdef __cplusplus
+#define OMNI_ALIGNAS(n) alignas(n)
 extern "C" {
+#else
+#define OMNI_ALIGNAS(n) _Alignas(n)
 #endif
 
 typedef enum {
@@ -96,6 +106,17 @@ int32_t omni_sparse_mla_num_splits(const omni_mla_desc_t *desc);
 int32_t omni_sparse_mla_num_launches(const omni_mla_desc_t *desc);
 
 /*
+ * The split-KV plan as a pure function of its inputs (no device needed; what
+ * omni_sparse_mla_num_splits / num_launches compute after asking the current device):
+ * partitions per request for this descriptor on a device with `sm_count` SMs on which
+ * `resident_merge_clusters` clusters of two CTA pairs of the paired-CTA kernel can be resident
+ * at once (33 on a 148-SM B200), and, through num_launches if non-NULL, the kernels one decode
+ * call launches.  Returns 0 on a bad descriptor or non-positive sm_count.
+ */
+int32_t omni_sparse_mla_plan_query(const omni_mla_desc_t *desc, int32_t sm_count,
+                                   int32_t resident_merge_clusters, int32_t *num_launches);
+
+/*
  * Bytes of device workspace omni_sparse_mla_decode needs for this descriptor: room for the
  * fp32 partial outputs and partial log-sum-exps of every (request, split) and for the
  * arrival counters of the in-kernel merge.  Returns 0 on a bad descriptor.  The workspace
@@ -135,6 +156,34 @@ omni_status_t omni_sparse_mla_decode(const omni_mla_desc_t *desc, const void *q,
                                      const int32_t *sel_idx, const int32_t *sel_len, void *out,
                                      float *lse, void *workspace, size_t workspace_bytes,
                                      int32_t *device_status, void *stream);
+
+/*
+ * The same decode call in two halves, for callers that issue it every step on the same
+ * buffers (no counterpart in the paper: host-side packaging of omni_sparse_mla_decode).
+ * omni_sparse_mla_plan_init does, once, everything that depends only on the descriptor, the
+ * q buffer and the KV pool: the argument checks on those, the split-KV plan, the choice of
+ * kernel and merge path, the tensor-map encodings.  It writes the result into `plan`, memory
+ * the caller owns (64-byte aligned; plain data: it may be copied, and needs no clean-up).
+ * omni_sparse_mla_decode_planned then takes the per-step pointers, checks them, and launches:
+ * no table look-up, no lock, no device query beyond "is the plan's device current".
+ * Results are those of omni_sparse_mla_decode with the same arguments, bit for bit.
+ *
+ * A plan stays valid while q and kv_cache keep their addresses and sizes and the descriptor
+ * is unchanged; it belongs to the device that was current in plan_init (OMNI_ERR_CUDA from the
+ * planned call if another device is current).  A plan that plan_init did not complete is
+ * rejected with OMNI_ERR_SHAPE.  workspace / workspace_bytes, device_status and stream are as
+ * in omni_sparse_mla_decode; the workspace size is omni_sparse_mla_workspace_bytes(desc).
+ */
+typedef struct {
+    OMNI_ALIGNAS(64) unsigned char opaque[1024];
+} omni_mla_plan_t;
+omni_status_t omni_sparse_mla_plan_init(const omni_mla_desc_t *desc, const void *q,
+                                        const void *kv_cache, omni_mla_plan_t *plan);
+omni_status_t omni_sparse_mla_decode_planned(const omni_mla_plan_t *plan, const int32_t *page_table,
+                                             const int32_t *sel_idx, const int32_t *sel_len,
+                                             void *out, float *lse, void *workspace,
+                                             size_t workspace_bytes, int32_t *device_status,
+                                             void *stream);
 
 /*
  * The same operation with the index set of Eq. 2 of the paper (attention sink + recent

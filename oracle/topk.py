@@ -4,7 +4,9 @@ The paper's own index set is the sink + recent rule of Eq. 2; a token-level vari
 with "the k tokens of highest score".  The definition used here: order the positions 0..M-1 of a
 request by score, highest first, where NaN ranks below every number and -0 below +0, equal
 scores by increasing position; keep the first min(k, M) positions of that order and report them
-in increasing order of position.
+in increasing order of position.  All NaNs are equal to one another whatever their sign bit or
+payload (the sign distinction applies to numbers only, where it separates -0 from +0), so among
+NaNs the lower position wins.
 """
 from __future__ import annotations
 
@@ -20,7 +22,7 @@ def topk_positions(scores, M: int, k: int) -> np.ndarray:
         return np.zeros(0, dtype=np.int32)
     is_num = ~np.isnan(s)
     value = np.where(is_num, s, np.float32(0)).astype(np.float64)
-    positive_sign = ~np.signbit(s)
+    positive_sign = np.where(is_num, ~np.signbit(s), True)      # the sign key orders numbers only
     # np.lexsort sorts by its LAST key first; every key ascending
     order = np.lexsort((np.arange(M), ~positive_sign, -value, ~is_num))
     return np.sort(order[:take]).astype(np.int32)

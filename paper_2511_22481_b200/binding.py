@@ -33,6 +33,7 @@ EXPORTS = (
     "omni_sparse_mla_validate", "omni_sparse_mla_resolve_rows",
     "omni_sparse_mla_host_staging_bytes", "omni_sparse_mla_decode_host",
     "omni_sparse_mla_set_profile_events", "omni_sparse_mla_decode_static",
+    "omni_sparse_mla_plan_init", "omni_sparse_mla_decode_planned", "omni_sparse_mla_plan_query",
 )
 
 
@@ -106,6 +107,12 @@ def load() -> ctypes.CDLL:
     lib.omni_sparse_mla_decode_host.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp, sz, vp, vp]
     lib.omni_sparse_mla_decode_static.restype = ctypes.c_int
     lib.omni_sparse_mla_decode_static.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.omni_sparse_mla_plan_query.restype = i32
+    lib.omni_sparse_mla_plan_query.argtypes = [dp, i32, i32, ctypes.POINTER(ctypes.c_int32)]
+    lib.omni_sparse_mla_plan_init.restype = ctypes.c_int
+    lib.omni_sparse_mla_plan_init.argtypes = [dp, vp, vp, vp]
+    lib.omni_sparse_mla_decode_planned.restype = ctypes.c_int
+    lib.omni_sparse_mla_decode_planned.argtypes = [vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
     lib.omni_sparse_mla_set_profile_events.restype = None
     lib.omni_sparse_mla_set_profile_events.argtypes = [vp, vp]
     _lib = lib
@@ -156,6 +163,14 @@ def omni_sparse_mla_num_splits(desc: OmniDesc) -> int:
 
 def omni_sparse_mla_num_launches(desc: OmniDesc) -> int:
     return int(load().omni_sparse_mla_num_launches(ctypes.byref(desc)))
+
+
+def omni_sparse_mla_plan_query(desc: OmniDesc, sm_count: int, resident_merge_clusters: int):
+    """(splits per request, launches per call) on a device description; needs no GPU."""
+    launches = ctypes.c_int32(0)
+    splits = int(load().omni_sparse_mla_plan_query(ctypes.byref(desc), int(sm_count), int(resident_merge_clusters),
+                                                   ctypes.byref(launches)))
+    return splits, int(launches.value)
 
 
 def omni_sparse_mla_workspace_bytes(desc: OmniDesc) -> int:
@@ -240,6 +255,61 @@ def omni_sparse_mla_decode_rolling(desc, q, kv_cache, page_table, ctx_len, n_sin
         None if workspace is None else ctypes.c_void_p(workspace.data_ptr()), ws_bytes,
         _ptr(device_status, torch.int32, "cuda", "device_status"), _stream(stream))
     _check(code, "omni_sparse_mla_decode_rolling")
+
+
+OMNI_PLAN_BYTES = 1024
+
+
+class LaunchPlan:
+    """Caller-owned storage of an ``omni_mla_plan_t`` (64-byte aligned host memory)."""
+
+    def __init__(self):
+        self._raw = ctypes.create_string_buffer(OMNI_PLAN_BYTES + 64)
+        base = ctypes.addressof(self._raw)
+        self.address = (base + 63) & ~63
+        self.ptr = ctypes.c_void_p(self.address)
+
+
+def omni_sparse_mla_plan_init(desc, q, kv_cache) -> LaunchPlan:
+    """Everything of a decode call that depends only on the descriptor, q and the pool, done once."""
+    plan = LaunchPlan()
+    code = load().omni_sparse_mla_plan_init(
+        ctypes.byref(desc), _ptr(q, torch.bfloat16, "cuda", "q"),
+        _ptr(kv_cache, torch.bfloat16, "cuda", "kv_cache"), plan.ptr)
+    _check(code, "omni_sparse_mla_plan_init")
+    return plan
+
+
+def omni_sparse_mla_decode_planned(plan, page_table, sel_idx, sel_len, out, lse, workspace=None,
+                                   device_status=None, stream=None) -> None:
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    code = load().omni_sparse_mla_decode_planned(
+        plan.ptr, _ptr(page_table, torch.int32, "cuda", "page_table"),
+        _ptr(sel_idx, torch.int32, "cuda", "sel_idx"), _ptr(sel_len, torch.int32, "cuda", "sel_len"),
+        _ptr(out, torch.bfloat16, "cuda", "out"), _ptr(lse, torch.float32, "cuda", "lse"),
+        None if workspace is None else ctypes.c_void_p(workspace.data_ptr()), ws_bytes,
+        _ptr(device_status, torch.int32, "cuda", "device_status"), _stream(stream))
+    _check(code, "omni_sparse_mla_decode_planned")
+
+
+def bind_planned(plan, page_table, sel_idx, sel_len, out, lse, workspace=None, device_status=None, stream=None):
+    """The planned decode call with its arguments marshalled once: returns a function of no
+    arguments that makes the C call (for loops that repeat one call on fixed buffers; the
+    tensors must stay alive and in place, and the stream is the one given here)."""
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    fn = load().omni_sparse_mla_decode_planned
+    args = (plan.ptr, _ptr(page_table, torch.int32, "cuda", "page_table"),
+            _ptr(sel_idx, torch.int32, "cuda", "sel_idx"), _ptr(sel_len, torch.int32, "cuda", "sel_len"),
+            _ptr(out, torch.bfloat16, "cuda", "out"), _ptr(lse, torch.float32, "cuda", "lse"),
+            None if workspace is None else ctypes.c_void_p(workspace.data_ptr()), ctypes.c_size_t(ws_bytes),
+            _ptr(device_status, torch.int32, "cuda", "device_status"), _stream(stream))
+    keep = (plan, page_table, sel_idx, sel_len, out, lse, workspace, device_status)
+
+    def call(_keep=keep):
+        code = fn(*args)
+        if code != OMNI_OK:
+            raise OmniError(code, "omni_sparse_mla_decode_planned")
+    return call
 
 
 OMNI_STATIC_SCRATCH_BYTES = 32 * 1024 * 1024

@@ -21,6 +21,7 @@ cudaEvent_t g_profile_before = nullptr, g_profile_after = nullptr;
 struct DeviceInfo {
     int sm_count = 0;
     int cc_major = 0;
+    int index = -1;
     bool ok = false;
 };
 
@@ -41,6 +42,7 @@ const DeviceInfo &device_info()
             cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) == cudaSuccess) {
             info[dev].sm_count = sms;
             info[dev].cc_major = major;
+            info[dev].index = dev;
             info[dev].ok = true;
         }
     }
@@ -76,10 +78,12 @@ int units_per_request(const omni_mla_desc_t *d)
 
 // Two splits of a request can be merged inside a cluster of two CTA pairs as long as all those
 // clusters are resident at once.
-bool merge_in_cluster(const omni_mla_desc_t *d, int splits)
+bool merge_in_cluster(const omni_mla_desc_t *d, int splits, int resident_merge_clusters = -1)
 {
-    return splits == 2 && use_pair_kernel(d) && !(d->flags & (OMNI_FLAG_FUSED_MERGE | OMNI_FLAG_NO_CLUSTER_MERGE)) &&
-           d->batch <= tc2_max_merge_clusters();
+    if (!(splits == 2 && use_pair_kernel(d) && !(d->flags & (OMNI_FLAG_FUSED_MERGE | OMNI_FLAG_NO_CLUSTER_MERGE))))
+        return false;
+    if (resident_merge_clusters < 0) resident_merge_clusters = tc2_max_merge_clusters();
+    return d->batch <= resident_merge_clusters;
 }
 
 // Pick the number of split-KV partitions per request.  The kernel's work units run in waves over
@@ -90,7 +94,7 @@ bool merge_in_cluster(const omni_mla_desc_t *d, int splits)
 // they stay in L2), and so does the merge kernel at the end.  Two splits merged inside a
 // cluster of two CTA pairs avoid the partial results and pay about 5 for the exchange.
 // Minimise waves * (granules per unit + fixed parts) + merge.
-int choose_splits(const omni_mla_desc_t *d, int sm_count)
+int choose_splits(const omni_mla_desc_t *d, int sm_count, int resident_merge_clusters = -1)
 {
     if (d->num_splits >= 1) return d->num_splits;
     if (sm_count <= 0) sm_count = 148;
@@ -106,7 +110,7 @@ int choose_splits(const omni_mla_desc_t *d, int sm_count)
         long cost;
         if (s == 1)
             cost = waves * (per + 6);
-        else if (merge_in_cluster(d, s))
+        else if (merge_in_cluster(d, s, resident_merge_clusters))
             cost = waves * (per + 6) + 5;
         else
             cost = waves * (per + 6 + (waves > 1 ? 6 : 2)) + 6;     // partial results stay in L2 within one wave
@@ -235,24 +239,98 @@ int32_t omni_sparse_mla_num_launches(const omni_mla_desc_t *desc)
     return n;
 }
 
+int32_t omni_sparse_mla_plan_query(const omni_mla_desc_t *desc, int32_t sm_count, int32_t resident_merge_clusters,
+                                   int32_t *num_launches)
+{
+    if (!desc_ok(desc) || sm_count < 1 || resident_merge_clusters < 0) return 0;
+    const int s = choose_splits(desc, sm_count, resident_merge_clusters);
+    if (num_launches) {
+        int n = 1 + ((desc->flags & OMNI_FLAG_VALIDATE) ? 1 : 0);
+        if (s > 1 && !merge_in_cluster(desc, s, resident_merge_clusters) &&
+            !(use_pair_kernel(desc) && (desc->flags & OMNI_FLAG_FUSED_MERGE)))
+            ++n;
+        *num_launches = n;
+    }
+    return s;
+}
+
 size_t omni_sparse_mla_workspace_bytes(const omni_mla_desc_t *desc)
 {
     if (!desc_ok(desc)) return 0;
     return workspace_need(desc, choose_splits(desc, device_info().sm_count));
 }
 
-// Shared by the two decode entry points: the selection is an index list (sel_idx, sel_len) or,
-// with sel_idx == nullptr, Eq. 2's ranges (ctx_len, n_sink, n_recent).
-static omni_status_t decode_impl(const omni_mla_desc_t *desc, const void *q, const void *kv_cache,
-                                 const int32_t *page_table, const int32_t *sel_idx,
-                                 const int32_t *sel_len, const int32_t *ctx_len, int32_t n_sink,
-                                 int32_t n_recent, bool rolling, void *out, float *lse, void *workspace,
-                                 size_t workspace_bytes, int32_t *device_status, void *stream_)
+// Everything about a decode call that depends only on the descriptor, q and the pool: which
+// kernel, the split plan, workspace carving, tensor maps.  The ordinary entry points build
+// one per call (maps come from the cache); omni_sparse_mla_plan_init stores one in caller
+// memory so that omni_sparse_mla_decode_planned only fills in pointers and launches.
+constexpr uint32_t kPlanMagic = 0x4c504d4fu;
+struct LaunchPlan {
+    uint32_t magic;
+    int32_t kernel;            // 0 plain-FMA, 1 single-CTA tensor-core, 2 paired-CTA tensor-core
+    int32_t splits;
+    int32_t cluster_merge, longest_first, fused_merge;
+    int32_t device;
+    size_t need, part_out, part_lse, counters;
+    omni_mla_desc_t desc;
+    const void *q, *kv;
+    alignas(64) CUtensorMap maps[4];
+};
+static_assert(sizeof(LaunchPlan) <= sizeof(omni_mla_plan_t), "plan does not fit its public container");
+static_assert(alignof(LaunchPlan) <= 64, "plan alignment");
+
+static omni_status_t build_plan(const omni_mla_desc_t *desc, const void *q, const void *kv_cache, bool cached_maps,
+                                LaunchPlan *plan)
+{
+    if (!desc || !q || !kv_cache) return OMNI_ERR_NULL;
+    if (!desc_ok(desc)) return OMNI_ERR_SHAPE;
+    if (!aligned(q, 16) || !aligned(kv_cache, 128)) return OMNI_ERR_ALIGN;
+    const DeviceInfo &dev = device_info();
+    if (!dev.ok) return OMNI_ERR_CUDA;
+    if (dev.cc_major != 10) return OMNI_ERR_ARCH;
+    plan->desc = *desc;
+    plan->q = q;
+    plan->kv = kv_cache;
+    plan->device = dev.index;
+    plan->kernel = (desc->flags & OMNI_FLAG_SIMT) ? 0 : use_pair_kernel(desc) ? 2 : 1;
+    const int splits = choose_splits(desc, dev.sm_count);
+    plan->splits = splits;
+    plan->part_out = part_out_bytes(desc, splits);
+    plan->part_lse = part_lse_bytes(desc, splits);
+    plan->counters = counter_bytes(desc);
+    plan->need = workspace_need(desc, splits);
+    // Two splits of a request can be merged inside a cluster of two CTA pairs, without partial
+    // results in global memory, as long as all those clusters are resident at once.
+    plan->cluster_merge = merge_in_cluster(desc, splits) ? 1 : 0;
+    plan->fused_merge = (splits > 1 && merge_in_kernel(desc)) ? 1 : 0;
+    // several waves of work units: start the longest requests first (the kernel ranks them itself)
+    plan->longest_first = (plan->kernel == 2 && !plan->cluster_merge && desc->batch <= 256 &&
+                           (long)desc->batch * splits > dev.sm_count / 2)
+                              ? 1
+                              : 0;
+    DecodeParams shape = {};
+    shape.q = static_cast<const __nv_bfloat16 *>(q);
+    shape.kv = static_cast<const __nv_bfloat16 *>(kv_cache);
+    shape.num_pages = desc->num_pages;
+    shape.batch = desc->batch;
+    shape.heads = desc->num_heads;
+    if (plan->kernel == 2) {
+        if (!tc2_prepare_device() || !tc2_make_maps(shape, plan->maps, cached_maps)) return OMNI_ERR_CUDA;
+    } else if (plan->kernel == 1) {
+        if (!tc_prepare_device() || !tc_make_maps(shape, plan->maps, cached_maps)) return OMNI_ERR_CUDA;
+    }
+    plan->magic = kPlanMagic;
+    return OMNI_OK;
+}
+
+// Checks of the per-step arguments that need no device.
+static omni_status_t check_step_args(const omni_mla_desc_t *desc, const int32_t *page_table, const int32_t *sel_idx,
+                                     const int32_t *sel_len, const int32_t *ctx_len, int32_t n_sink, int32_t n_recent,
+                                     bool rolling, const void *out, const float *lse)
 {
     const bool ranges = sel_idx == nullptr;
-    if (!desc || !q || !kv_cache || !page_table || !out || !lse) return OMNI_ERR_NULL;
+    if (!page_table || !out || !lse) return OMNI_ERR_NULL;
     if (ranges ? !ctx_len : !sel_len) return OMNI_ERR_NULL;
-    if (!desc_ok(desc)) return OMNI_ERR_SHAPE;
     if (ranges) {
         // max_sel bounds the selection size the split plan is made for
         if (n_sink < 0 || n_recent < 0) return OMNI_ERR_SHAPE;
@@ -263,18 +341,28 @@ static omni_status_t decode_impl(const omni_mla_desc_t *desc, const void *q, con
         if (rolling && (int64_t)desc->max_pages_per_req < rolling_sink_pages(n_sink) + rolling_ring_pages(n_recent))
             return OMNI_ERR_SHAPE;
     }
-    if (!aligned(q, 16) || !aligned(kv_cache, 128) || !aligned(out, 16) || !aligned(lse, 4) ||
-        !aligned(page_table, 4) || !aligned(sel_idx, 4) || !aligned(sel_len, 4) || !aligned(ctx_len, 4))
+    if (!aligned(out, 16) || !aligned(lse, 4) || !aligned(page_table, 4) || !aligned(sel_idx, 4) || !aligned(sel_len, 4) ||
+        !aligned(ctx_len, 4))
         return OMNI_ERR_ALIGN;
-    const DeviceInfo &dev = device_info();
-    if (!dev.ok) return OMNI_ERR_CUDA;
-    if (dev.cc_major != 10) return OMNI_ERR_ARCH;
-    const int splits = choose_splits(desc, dev.sm_count);
-    const size_t need = workspace_need(desc, splits);
+    return OMNI_OK;
+}
+
+// The per-call half: pointer checks, workspace carving, launches.  The selection is an index
+// list (sel_idx, sel_len) or, with sel_idx == nullptr, Eq. 2's ranges (ctx_len, n_sink, n_recent).
+static omni_status_t run_plan(const LaunchPlan &plan, const int32_t *page_table, const int32_t *sel_idx,
+                              const int32_t *sel_len, const int32_t *ctx_len, int32_t n_sink, int32_t n_recent,
+                              bool rolling, void *out, float *lse, void *workspace, size_t workspace_bytes,
+                              int32_t *device_status, void *stream_)
+{
+    const omni_mla_desc_t *desc = &plan.desc;
+    const bool ranges = sel_idx == nullptr;
+    omni_status_t args = check_step_args(desc, page_table, sel_idx, sel_len, ctx_len, n_sink, n_recent, rolling, out, lse);
+    if (args != OMNI_OK) return args;
+    const int splits = plan.splits;
     if (splits > 1) {
         if (!workspace) return OMNI_ERR_NULL;
         if (!aligned(workspace, 256)) return OMNI_ERR_ALIGN;
-        if (workspace_bytes < need) return OMNI_ERR_WORKSPACE;
+        if (workspace_bytes < plan.need) return OMNI_ERR_WORKSPACE;
     }
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
 
@@ -284,8 +372,8 @@ static omni_status_t decode_impl(const omni_mla_desc_t *desc, const void *q, con
     }
 
     DecodeParams p;
-    p.q = static_cast<const __nv_bfloat16 *>(q);
-    p.kv = static_cast<const __nv_bfloat16 *>(kv_cache);
+    p.q = static_cast<const __nv_bfloat16 *>(plan.q);
+    p.kv = static_cast<const __nv_bfloat16 *>(plan.kv);
     p.page_table = page_table;
     p.sel_idx = sel_idx;
     p.sel_len = sel_len;
@@ -297,23 +385,14 @@ static omni_status_t decode_impl(const omni_mla_desc_t *desc, const void *q, con
     p.out = static_cast<__nv_bfloat16 *>(out);
     p.lse = lse;
     p.part_out = static_cast<float *>(workspace);
-    p.part_lse = splits > 1 ? reinterpret_cast<float *>(static_cast<char *>(workspace) + part_out_bytes(desc, splits))
-                            : nullptr;
+    p.part_lse = splits > 1 ? reinterpret_cast<float *>(static_cast<char *>(workspace) + plan.part_out) : nullptr;
     p.status = device_status;
     p.counters = nullptr;
-    p.cluster_merge = 0;
-    // Two splits of a request can be merged inside a cluster of two CTA pairs, without partial
-    // results in global memory, as long as all those clusters are resident at once.
-    if (merge_in_cluster(desc, splits)) p.cluster_merge = 1;
-    // several waves of work units: start the longest requests first (the kernel ranks them itself)
-    p.longest_first = (use_pair_kernel(desc) && !p.cluster_merge && desc->batch <= 256 &&
-                       (long)desc->batch * splits > dev.sm_count / 2)
-                          ? 1
-                          : 0;
-    if (splits > 1 && merge_in_kernel(desc)) {
-        p.counters = reinterpret_cast<int32_t *>(static_cast<char *>(workspace) + part_out_bytes(desc, splits) +
-                                                 part_lse_bytes(desc, splits));
-        if (cudaMemsetAsync(p.counters, 0, counter_bytes(desc), stream) != cudaSuccess) return OMNI_ERR_CUDA;
+    p.cluster_merge = plan.cluster_merge;
+    p.longest_first = plan.longest_first;
+    if (plan.fused_merge) {
+        p.counters = reinterpret_cast<int32_t *>(static_cast<char *>(workspace) + plan.part_out + plan.part_lse);
+        if (cudaMemsetAsync(p.counters, 0, plan.counters, stream) != cudaSuccess) return OMNI_ERR_CUDA;
     }
     p.num_pages = desc->num_pages;
     p.batch = desc->batch;
@@ -323,20 +402,67 @@ static omni_status_t decode_impl(const omni_mla_desc_t *desc, const void *q, con
     p.splits = splits;
     p.scale_log2 = desc->softmax_scale * kLog2e;
 
-    if (g_profile_before && g_profile_after) cudaEventRecord(g_profile_before, stream);
-    if (desc->flags & OMNI_FLAG_SIMT) {
+    const bool profile = g_profile_before && g_profile_after;
+    if (profile) cudaEventRecord(g_profile_before, stream);
+    omni_status_t st = OMNI_OK;
+    if (plan.kernel == 0) {
         const int grid = desc->batch * splits * units_per_request(desc);
         simt_decode_kernel<<<grid, kSimtWarps * 32, 0, stream>>>(p);
-        if (cudaPeekAtLastError() != cudaSuccess) return OMNI_ERR_CUDA;
+        if (cudaPeekAtLastError() != cudaSuccess) st = OMNI_ERR_CUDA;
     } else {
-        omni_status_t st = use_pair_kernel(desc) ? launch_tc2_decode(p, stream) : launch_tc_decode(p, stream);
-        if (st != OMNI_OK) return st;
+        st = plan.kernel == 2 ? tc2_launch(plan.maps, p, stream) : tc_launch(plan.maps, p, stream);
     }
-    if (g_profile_before && g_profile_after) cudaEventRecord(g_profile_after, stream);
+    if (st != OMNI_OK) return st;
+    if (profile) cudaEventRecord(g_profile_after, stream);
     if (splits > 1 && p.counters == nullptr && !p.cluster_merge)
         return launch_combine(desc->batch, desc->num_heads, splits, p.part_out, p.part_lse, nullptr,
                               out, lse, stream);
     return OMNI_OK;
+}
+
+static omni_status_t decode_impl(const omni_mla_desc_t *desc, const void *q, const void *kv_cache,
+                                 const int32_t *page_table, const int32_t *sel_idx,
+                                 const int32_t *sel_len, const int32_t *ctx_len, int32_t n_sink,
+                                 int32_t n_recent, bool rolling, void *out, float *lse, void *workspace,
+                                 size_t workspace_bytes, int32_t *device_status, void *stream)
+{
+    // everything the host can check is checked before the device is asked anything
+    if (!desc || !q || !kv_cache || !page_table || !out || !lse) return OMNI_ERR_NULL;
+    if (sel_idx == nullptr ? !ctx_len : !sel_len) return OMNI_ERR_NULL;
+    if (!desc_ok(desc)) return OMNI_ERR_SHAPE;
+    omni_status_t st = check_step_args(desc, page_table, sel_idx, sel_len, ctx_len, n_sink, n_recent, rolling, out, lse);
+    if (st == OMNI_OK && (!aligned(q, 16) || !aligned(kv_cache, 128))) st = OMNI_ERR_ALIGN;
+    if (st != OMNI_OK) return st;
+    LaunchPlan plan;
+    st = build_plan(desc, q, kv_cache, true, &plan);
+    if (st != OMNI_OK) return st;
+    return run_plan(plan, page_table, sel_idx, sel_len, ctx_len, n_sink, n_recent, rolling, out, lse, workspace,
+                    workspace_bytes, device_status, stream);
+}
+
+omni_status_t omni_sparse_mla_plan_init(const omni_mla_desc_t *desc, const void *q, const void *kv_cache,
+                                        omni_mla_plan_t *plan)
+{
+    if (!plan) return OMNI_ERR_NULL;
+    if (!aligned(plan, 64)) return OMNI_ERR_ALIGN;
+    LaunchPlan *lp = reinterpret_cast<LaunchPlan *>(plan);
+    lp->magic = 0;
+    return build_plan(desc, q, kv_cache, false, lp);
+}
+
+omni_status_t omni_sparse_mla_decode_planned(const omni_mla_plan_t *plan, const int32_t *page_table,
+                                             const int32_t *sel_idx, const int32_t *sel_len, void *out,
+                                             float *lse, void *workspace, size_t workspace_bytes,
+                                             int32_t *device_status, void *stream)
+{
+    if (!plan || !sel_idx) return OMNI_ERR_NULL;
+    if (!aligned(plan, 64)) return OMNI_ERR_ALIGN;
+    const LaunchPlan *lp = reinterpret_cast<const LaunchPlan *>(plan);
+    if (lp->magic != kPlanMagic) return OMNI_ERR_SHAPE;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev != lp->device) return OMNI_ERR_CUDA;
+    return run_plan(*lp, page_table, sel_idx, sel_len, nullptr, 0, 0, false, out, lse, workspace, workspace_bytes,
+                    device_status, stream);
 }
 
 omni_status_t omni_sparse_mla_decode(const omni_mla_desc_t *desc, const void *q,
@@ -441,25 +567,6 @@ omni_status_t omni_sparse_mla_resolve_rows(const omni_mla_desc_t *desc,
                           static_cast<cudaStream_t>(stream));
 }
 
-#ifdef OMNI_TRACE
-// development builds only: copies the timeline records of the last launches to the host
-int omni_trace_read(void *host, size_t bytes)
-{
-    if (bytes > sizeof(unsigned long long) * 2 * kTraceWarps * kTraceEvents) return 1;
-    return cudaMemcpyFromSymbol(host, g_trace, bytes) == cudaSuccess ? 0 : 2;
-}
-int omni_span_read(void *host, size_t bytes)
-{
-    if (bytes > sizeof(unsigned long long) * 2048 * 8) return 1;
-    return cudaMemcpyFromSymbol(host, g_span, bytes) == cudaSuccess ? 0 : 2;
-}
-int omni_trace_clear(void)
-{
-    void *ptr = nullptr;
-    if (cudaGetSymbolAddress(&ptr, g_trace) != cudaSuccess) return 2;
-    return cudaMemset(ptr, 0, sizeof(unsigned long long) * 2 * kTraceWarps * kTraceEvents) == cudaSuccess ? 0 : 2;
-}
-#endif
 
 // The host-buffer entry point splits a large batch into two parts so that the second part's
 // host-to-device copies run under the first half's kernel, and the first half's device-to-host

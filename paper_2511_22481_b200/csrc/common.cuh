@@ -114,6 +114,14 @@ __device__ __forceinline__ Selection load_selection(const DecodeParams &p, int b
     return s;
 }
 
+// Whether entry value t is range padding ("no token") rather than a position the caller wrote:
+// only the range form pads, so in an index list -2 is a negative position like any other and
+// breaks the index contract.
+__device__ __forceinline__ bool is_padding(const Selection &s, int32_t t)
+{
+    return s.list == nullptr && t == kSelectionPad;
+}
+
 __device__ __forceinline__ int32_t selection_at(const Selection &s, int j)
 {
     if (s.list != nullptr) return __ldg(s.list + j);
@@ -138,35 +146,5 @@ __device__ __forceinline__ void flag_status(int32_t *status, int32_t bits)
 {
     if (status != nullptr) atomicOr(status, bits);
 }
-
-// Timeline probe of development builds (-DOMNI_TRACE; never defined in the shipped library):
-// lane 0 of every warp of the first two CTAs appends (time in ns, tile, event id) records that
-// omni_trace_read copies out.
-#ifdef OMNI_TRACE
-constexpr int kTraceWarps = 12, kTraceEvents = 1024;
-__device__ unsigned long long g_trace[2][kTraceWarps][kTraceEvents];
-__device__ __forceinline__ unsigned long long trace_time_ns()
-{
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-__device__ unsigned long long g_span[2048][8];   // per CTA: entry, set-up done, last P V retired, exit, merge phases
-#define OMNI_SPAN(slot)                                                                             \
-    do {                                                                                            \
-        if (threadIdx.x == 64 && blockIdx.x < 2048) g_span[blockIdx.x][slot] = trace_time_ns();     \
-    } while (0)
-#define OMNI_TRACE_DECL int trace_n = 0;
-#define OMNI_STAMP(ev, tile)                                                                        \
-    do {                                                                                            \
-        if (blockIdx.x < 2 && (threadIdx.x & 31) == 0 && trace_n < kTraceEvents)                    \
-            g_trace[blockIdx.x][threadIdx.x >> 5][trace_n++] =                                      \
-                (trace_time_ns() << 20) | ((unsigned long long)((tile) & 0xfff) << 8) | (ev);       \
-    } while (0)
-#else
-#define OMNI_TRACE_DECL
-#define OMNI_STAMP(ev, tile)
-#define OMNI_SPAN(slot)
-#endif
 
 }  // namespace omni

@@ -59,7 +59,7 @@ __global__ void __launch_bounds__(kSimtWarps * 32) simt_decode_kernel(DecodePara
     const int32_t *pt = p.page_table + (size_t)b * p.max_pages;
     for (int j = begin; j < end; ++j) {
         const int32_t t = selection_at(selection, j);
-        if (t == kSelectionPad) continue;
+        if (is_padding(selection, t)) continue;
         const int64_t row = resolve_row(pt, t, p.max_pages, p.num_pages);
         if (row < 0) {
             if (lane == 0) flag_status(p.status, OMNI_DEV_BAD_INDEX);

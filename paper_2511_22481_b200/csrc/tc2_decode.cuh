@@ -81,6 +81,7 @@ struct C2Control {
     uint32_t tmem_base;
     uint32_t abort;
     uint32_t merge_flag;
+    uint32_t xfail;                      // cluster merge: some wait of this CTA ran out (decided CTA-wide)
     int32_t k_progress;                  // tiles whose K loads the producer has started (L2 prefetch pacing)
     uint64_t recv_bar;                   // cluster merge: the partner's block has arrived
     uint64_t ready_bar;                  // cluster merge: the partner's main loop is over
@@ -257,7 +258,7 @@ __device__ __forceinline__ void tc_commit_pair_elect(uint64_t *bar, uint16_t bot
 // Called by every thread of the CTA after the main loop.
 __device__ __forceinline__ void cluster_merge_exchange(const DecodeParams &p, C2Control *ctl, uint8_t *smem,
                                                        uint32_t tmem, int b, int s, uint32_t crank, int h0,
-                                                       int head_rows, bool active, float cm_lse, float cm_inv)
+                                                       int head_rows, bool active, bool main_ok, float cm_lse, float cm_inv)
 {
     constexpr uint32_t kSliceBytes = 256 * 4;            // half of a row's value columns, fp32
     constexpr uint32_t kPitch = kSliceBytes + 16;        // row-per-lane 16-byte accesses do not conflict
@@ -273,6 +274,11 @@ __device__ __forceinline__ void cluster_merge_exchange(const DecodeParams &p, C2
     const uint32_t partner = crank ^ 2u;
     // an empty split never ran a main loop: its shared memory is free from the start
     if (!active && warp == 2 && lane == 0) mbar_arrive_cluster(map_to_rank(smem_u32(&ctl->ready_bar), partner));
+    // Whether anything went wrong is decided for the whole CTA, never per warp: all eight warps
+    // pass the same named barriers below and then go on or leave together.  A warp whose main
+    // loop ran into a bounded wait says so here; the decision is read after the next barrier.
+    volatile uint32_t *xfail = &ctl->xfail;
+    if (!main_ok && lane == 0) *xfail = 1u;
 
     // this thread's 128 value columns are finished by split `part / 2`
     uint8_t *tile = ((part >> 1) == s ? keep : send) + (size_t)row * kPitch + (part & 1) * 512;
@@ -301,11 +307,16 @@ __device__ __forceinline__ void cluster_merge_exchange(const DecodeParams &p, C2
     tc_fence_before();
     fence_async_smem();                                   // the bulk copy reads what the threads wrote
     asm volatile("bar.sync 1, 256;" ::: "memory");         // the eight softmax warps
-    bool ok = true;
+    const bool main_failed = *xfail != 0u;
     if (warp == 2) {
-        ok = mbar_wait(&ctl->ready_bar, 0);               // the partner's operand tiles are dead
-        ok = __all_sync(0xffffffffu, ok);
-        if (ok && lane == 0) {
+        // A CTA whose main loop gave up never told its partner that its operand tiles are dead
+        // (that arrive sits at the end of the main loop).  It does so now, and it still sends a
+        // block (of unspecified contents: the status word already says so), so that every wait
+        // of the healthy partner ends and both CTAs finish together.
+        if (main_failed && active && lane == 0) mbar_arrive_cluster(map_to_rank(smem_u32(&ctl->ready_bar), partner));
+        bool ready = mbar_wait(&ctl->ready_bar, 0);       // the partner's operand tiles are dead
+        ready = __all_sync(0xffffffffu, ready);
+        if (ready && lane == 0) {
             mbar_expect_tx(&ctl->recv_bar, kBlockBytes);
             const uint32_t dst = map_to_rank(smem_u32(recv), partner);
             const uint32_t bar = map_to_rank(smem_u32(&ctl->recv_bar), partner);
@@ -313,12 +324,17 @@ __device__ __forceinline__ void cluster_merge_exchange(const DecodeParams &p, C2
                          ::"r"(dst), "r"(smem_u32(send)), "r"(kBlockBytes), "r"(bar)
                          : "memory");
         }
+        if (!ready && lane == 0) *xfail = 1u;
     }
-    ok = ok && mbar_wait(&ctl->recv_bar, 0);
-    ok = __all_sync(0xffffffffu, ok);
-    if (!ok) {
-        if (lane == 0) flag_status(p.status, OMNI_DEV_TIMEOUT | OMNI_DEV_ROLE_SOFTMAX);
-        return;
+    {
+        bool got = mbar_wait(&ctl->recv_bar, 0);
+        got = __all_sync(0xffffffffu, got);
+        if (!got && lane == 0) *xfail = 1u;
+    }
+    asm volatile("bar.sync 1, 256;" ::: "memory");         // every warp's verdict is in
+    if (*xfail != 0u) {
+        if (warp == 2 && lane == 0) flag_status(p.status, OMNI_DEV_TIMEOUT | OMNI_DEV_ROLE_SOFTMAX);
+        return;                                            // all eight warps leave here together
     }
     // weights of the two splits per head row (in place of the log-sum-exps), final log-sum-exp
     if (part == 0) {
@@ -383,9 +399,6 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
     const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;  // warp-uniform
     const int h0 = (int)rank * kTcHeads;
     const int head_rows = min(kTcHeads, p.heads - h0);
-    OMNI_TRACE_DECL
-    OMNI_STAMP(0x04, 0);
-    OMNI_SPAN(0);
 
     // ---- set-up: barriers and tensor memory (nothing here touches global memory, so with a
     // programmatic dependent launch it overlaps the tail of the kernel before this one) --------
@@ -407,6 +420,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
         mbar_init(&ctl->recv_bar, 1);
         mbar_init(&ctl->ready_bar, 1);
         ctl->abort = 0;
+        ctl->xfail = 0;
         ctl->k_progress = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -474,8 +488,6 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
 
     const uint32_t tmem = ctl->tmem_base;
     volatile uint32_t *abort_flag = &ctl->abort;
-    OMNI_STAMP(0x01, 0);
-    OMNI_SPAN(1);
 
     const int32_t *pt = p.page_table + (size_t)b * p.max_pages;
 
@@ -502,7 +514,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
                           bool &contig_lo, bool &contig_hi, bool &any_bad) {
         const int j0 = begin + tile * kC2Tile + lane, j1 = j0 + 32;
         const bool ok0 = x.pg0 >= 0 && (int64_t)x.pg0 < p.num_pages, ok1 = x.pg1 >= 0 && (int64_t)x.pg1 < p.num_pages;
-        any_bad |= (j0 < end && !ok0 && x.t0 != kSelectionPad) || (j1 < end && !ok1 && x.t1 != kSelectionPad);
+        any_bad |= (j0 < end && !ok0 && !is_padding(selection, x.t0)) || (j1 < end && !ok1 && !is_padding(selection, x.t1));
         const int r0 = ok0 ? x.pg0 * kPage + x.t0 % kPage : -1, r1 = ok1 ? x.pg1 * kPage + x.t1 % kPage : -1;
         const uint32_t m0 = __ballot_sync(0xffffffffu, r0 >= 0), m1 = __ballot_sync(0xffffffffu, r1 >= 0);
         mask = (uint64_t)m0 | ((uint64_t)m1 << 32);
@@ -521,6 +533,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
 
     // what the cluster merge needs from the softmax warps after the main loop
     float cm_lse = -INFINITY, cm_inv = 0.f;
+    bool softmax_ok = true;              // false in a softmax warp whose main loop ran into a bounded wait
 
     if (!active) {
         // an empty split inside a merging cluster: no pipeline, but it takes part in the exchange
@@ -564,7 +577,6 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
             const uint32_t bar = map_to_rank(smem_u32(&ctl->k_full[st]), leader);
             if (lane == 0 && rank == 0) mbar_expect_tx(&ctl->k_full[st], 2 * kC2KBytes);
             __syncwarp();
-            OMNI_STAMP(0x10, i);
             const uint32_t dst = smem_base + kC2SmemK + st * kC2KBytes;
             const int own_row = rank ? row_hi : row_lo;
             bool gathered = false;
@@ -624,7 +636,6 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
             const uint32_t bar = map_to_rank(smem_u32(&ctl->v_full[st]), leader);
             if (lane == 0 && rank == 0) mbar_expect_tx(&ctl->v_full[st], 2 * kC2VBytes);
             __syncwarp();
-            OMNI_STAMP(0x50, i);
             const uint32_t dst = smem_base + kC2SmemV + st * kC2VBytes;
             bool gathered = false;
             if (contig) {
@@ -750,9 +761,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
                 good = __all_sync(0xffffffffu, good);
                 if (!good) return false;
                 tc_fence_after();
-                OMNI_STAMP(0x20, t);
                 issue_qk(kpar_tag, sbuf_tag);
-                OMNI_STAMP(0x28, t);
                 return true;
             };
             auto pv_tile = [&](auto par_tag, int i) -> bool {
@@ -761,9 +770,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
                 good = __all_sync(0xffffffffu, good);
                 if (!good) return false;
                 tc_fence_after();
-                OMNI_STAMP(0x30, i);
                 issue_pv(par_tag, i == 0);
-                OMNI_STAMP(0x38, i);
                 return true;
             };
             using I0 = std::integral_constant<int, 0>;
@@ -831,7 +838,6 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
             }
             tc_fence_after();
             uint32_t sv[16];
-            OMNI_STAMP(0x40, i);
             tc_ld16(tmem + lane_base + kC2ColS + 32 * sbuf + 16 * sub, sv);
             tc_wait_ld();
             tc_fence_before();
@@ -918,12 +924,9 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(buf ? p_full_leader1 : p_full_leader0);
-            OMNI_STAMP(0x43, i);
         }
         if (ok) {
             ok = mbar_wait(&ctl->pv_done[(tiles - 1) & 1], ((tiles - 1) >> 1) & 1);
-            OMNI_STAMP(0x48, 0);
-            OMNI_SPAN(2);
             ok = __all_sync(0xffffffffu, ok);
         }
         if (ok) {
@@ -1024,12 +1027,12 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
             }
             // with the in-kernel merge the partial results must be visible before this CTA is counted
             if (!final_out && p.counters != nullptr) __threadfence();
-            OMNI_STAMP(0x49, 0);
         }
         if (!ok && lane == 0) {
             flag_status(p.status, OMNI_DEV_TIMEOUT | OMNI_DEV_ROLE_SOFTMAX);
             *abort_flag = 1;
         }
+        softmax_ok = ok;
     }
 
     // ---- tear-down: nobody leaves while the other CTA may still touch this one's memory --
@@ -1037,7 +1040,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
         // a wait ran out: give copies that are still in flight time to land before anyone exits
         for (int i = 0; i < 200; ++i) __nanosleep(1000);
     }
-    if (p.cluster_merge) cluster_merge_exchange(p, ctl, smem, tmem, b, s, crank, h0, head_rows, active, cm_lse, cm_inv);
+    if (p.cluster_merge) cluster_merge_exchange(p, ctl, smem, tmem, b, s, crank, h0, head_rows, active, softmax_ok, cm_lse, cm_inv);
     tc_fence_before();
     __syncthreads();
     // Tensor memory was allocated for the pair, so it is released only when both CTAs are done
@@ -1058,11 +1061,8 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
     // before every CTA of the cluster has received its block
     if (p.cluster_merge) cluster_sync_relaxed();
     // ---- split merge by whichever CTA finishes a (request, head half) last ---------------
-    OMNI_STAMP(0x02, 0);
     if (p.splits > 1 && p.counters != nullptr)
         merge_if_last(p, b, (int)rank, 2, h0, head_rows, reinterpret_cast<float *>(smem), &ctl->merge_flag);
-    OMNI_STAMP(0x03, 0);
-    OMNI_SPAN(3);
 }
 
 // Clusters of two pairs (cluster merge) that can be resident at once on the current device, or 0.
@@ -1070,8 +1070,10 @@ inline int tc2_max_merge_clusters()
 {
     static int cached[64];
     static bool known[64] = {};
+    static std::mutex mu;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    std::lock_guard<std::mutex> lock(mu);
     if (!known[dev]) {
         int n = 0;
         if (cudaFuncSetAttribute(tc2_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kC2SmemBytes) == cudaSuccess) {
@@ -1097,22 +1099,35 @@ inline int tc2_max_merge_clusters()
     return cached[dev];
 }
 
-inline omni_status_t launch_tc2_decode(const DecodeParams &p, cudaStream_t stream)
+inline bool tc2_prepare_device()
 {
     static bool attr_set[64] = {};
+    static std::mutex mu;
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return OMNI_ERR_CUDA;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+    std::lock_guard<std::mutex> lock(mu);
     if (!attr_set[dev]) {
         if (cudaFuncSetAttribute(tc2_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kC2SmemBytes) !=
             cudaSuccess)
-            return OMNI_ERR_CUDA;
+            return false;
         attr_set[dev] = true;
     }
-    CUtensorMap q_map, kv_k_map, kv_v_map, kv_tile_map;
-    if (!make_panel_map(&kv_tile_map, p.kv, (uint64_t)p.num_pages * kPage, kTile, kPanels)) return OMNI_ERR_CUDA;
-    if (!make_panel_map(&q_map, p.q, (uint64_t)p.batch * p.heads, kTcHeads, kPanels)) return OMNI_ERR_CUDA;
-    if (!make_panel_map(&kv_k_map, p.kv, (uint64_t)p.num_pages * kPage, 32, kPanels)) return OMNI_ERR_CUDA;
-    if (!make_panel_map(&kv_v_map, p.kv, (uint64_t)p.num_pages * kPage, kTile, 4)) return OMNI_ERR_CUDA;
+    return true;
+}
+
+// maps[0] = q, maps[1] = K role boxes, maps[2] = V role boxes, maps[3] = whole pages
+inline bool tc2_make_maps(const DecodeParams &p, CUtensorMap *maps, bool cached)
+{
+    const uint64_t rows = (uint64_t)p.num_pages * kPage, qrows = (uint64_t)p.batch * p.heads;
+    if (cached)
+        return make_panel_map(&maps[0], p.q, qrows, kTcHeads, kPanels) && make_panel_map(&maps[1], p.kv, rows, 32, kPanels) &&
+               make_panel_map(&maps[2], p.kv, rows, kTile, 4) && make_panel_map(&maps[3], p.kv, rows, kTile, kPanels);
+    return encode_panel_map(&maps[0], p.q, qrows, kTcHeads, kPanels) && encode_panel_map(&maps[1], p.kv, rows, 32, kPanels) &&
+           encode_panel_map(&maps[2], p.kv, rows, kTile, 4) && encode_panel_map(&maps[3], p.kv, rows, kTile, kPanels);
+}
+
+inline omni_status_t tc2_launch(const CUtensorMap *maps, const DecodeParams &p, cudaStream_t stream)
+{
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(p.batch * p.splits * 2));
     cfg.blockDim = dim3(kC2Threads);
@@ -1129,7 +1144,7 @@ inline omni_status_t launch_tc2_decode(const DecodeParams &p, cudaStream_t strea
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, tc2_decode_kernel, q_map, kv_k_map, kv_v_map, kv_tile_map, p) == cudaSuccess
+    return cudaLaunchKernelEx(&cfg, tc2_decode_kernel, maps[0], maps[1], maps[2], maps[3], p) == cudaSuccess
                ? OMNI_OK
                : OMNI_ERR_CUDA;
 }

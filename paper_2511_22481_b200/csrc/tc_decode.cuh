@@ -393,11 +393,11 @@ tc_decode_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constan
             int64_t r0 = -1, r1 = -1;
             if (j0 < end) {
                 r0 = resolve_row(pt, t0, p.max_pages, p.num_pages);
-                any_bad |= (r0 < 0 && t0 != kSelectionPad);
+                any_bad |= (r0 < 0 && !is_padding(selection, t0));
             }
             if (j1 < end) {
                 r1 = resolve_row(pt, t1, p.max_pages, p.num_pages);
-                any_bad |= (r1 < 0 && t1 != kSelectionPad);
+                any_bad |= (r1 < 0 && !is_padding(selection, t1));
             }
             const uint32_t m0 = __ballot_sync(0xffffffffu, r0 >= 0), m1 = __ballot_sync(0xffffffffu, r1 >= 0);
             mask = (uint64_t)m0 | ((uint64_t)m1 << 32);
@@ -711,40 +711,44 @@ inline EncodeTiledFn encode_tiled_fn()
 }
 
 // Encoding a tensor map costs about a microsecond of host time and a decode step needs up to
-// five, more than the launch itself, so the most recent encodings are kept (a map depends only
-// on the base address and the sizes; nothing in it refers to a call).
+// four, more than the launch itself, so encodings are kept (a map depends only on the base
+// address and the sizes; nothing in it refers to a call).  Callers that must not pay even the
+// lookup build a plan once (omni_sparse_mla_plan_init), which stores the maps themselves.
+// The table is direct-mapped on a hash of the key and large enough for the maps of a few
+// hundred distinct pools (a model with one KV pool per layer uses three maps per layer); a
+// colliding key replaces the older entry.
 struct MapCacheEntry {
     const void *base;
     uint64_t rows;
     uint32_t box_rows, box_panels, kind;
+    bool used;
     CUtensorMap map;
 };
 
 inline bool cached_map(CUtensorMap *out, const void *base, uint64_t rows, uint32_t box_rows, uint32_t box_panels,
                        uint32_t kind, bool (*encode)(CUtensorMap *, const void *, uint64_t, uint32_t, uint32_t))
 {
-    constexpr int kEntries = 32;
+    constexpr uint32_t kEntries = 1024;
     static MapCacheEntry cache[kEntries];
-    static int used = 0, next = 0;
     static std::mutex mu;
+    uint64_t h = reinterpret_cast<uintptr_t>(base) * 0x9E3779B97F4A7C15ull;
+    h ^= (rows + 0x7F4A7C15ull) * 0xC2B2AE3D27D4EB4Full;
+    h ^= ((uint64_t)box_rows << 40) ^ ((uint64_t)box_panels << 20) ^ kind;
+    h *= 0x9E3779B97F4A7C15ull;
+    MapCacheEntry &e = cache[(h >> 40) % kEntries];
     std::lock_guard<std::mutex> lock(mu);
-    for (int i = 0; i < used; ++i) {
-        const MapCacheEntry &e = cache[i];
-        if (e.base == base && e.rows == rows && e.box_rows == box_rows && e.box_panels == box_panels && e.kind == kind) {
-            *out = e.map;
-            return true;
-        }
+    if (e.used && e.base == base && e.rows == rows && e.box_rows == box_rows && e.box_panels == box_panels && e.kind == kind) {
+        *out = e.map;
+        return true;
     }
     if (!encode(out, base, rows, box_rows, box_panels)) return false;
-    MapCacheEntry &e = cache[next];
     e.base = base;
     e.rows = rows;
     e.box_rows = box_rows;
     e.box_panels = box_panels;
     e.kind = kind;
     e.map = *out;
-    next = (next + 1) % kEntries;
-    if (used < kEntries) ++used;
+    e.used = true;
     return true;
 }
 
@@ -788,21 +792,37 @@ inline bool make_panel_map(CUtensorMap *map, const void *base, uint64_t rows, ui
     return cached_map(map, base, rows, box_rows, box_panels, 1, encode_panel_map);
 }
 
-inline omni_status_t launch_tc_decode(const DecodeParams &p, cudaStream_t stream)
+// Host side of a launch, in three steps so that a plan can do the first two once:
+// per-device kernel attributes, the tensor maps, the launch itself.
+inline bool tc_prepare_device()
 {
     static bool attr_set[64] = {};
+    static std::mutex mu;
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return OMNI_ERR_CUDA;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+    std::lock_guard<std::mutex> lock(mu);
     if (!attr_set[dev]) {
         if (cudaFuncSetAttribute(tc_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBytes) !=
             cudaSuccess)
-            return OMNI_ERR_CUDA;
+            return false;
         attr_set[dev] = true;
     }
-    CUtensorMap q_map, kv_map, kv_page_map;
-    if (!make_panel_map(&q_map, p.q, (uint64_t)p.batch * p.heads, kTcHeads, kPanels)) return OMNI_ERR_CUDA;
-    if (!make_row_map(&kv_map, p.kv, (uint64_t)p.num_pages * kPage, 1)) return OMNI_ERR_CUDA;
-    if (!make_panel_map(&kv_page_map, p.kv, (uint64_t)p.num_pages * kPage, kTile, kPanels)) return OMNI_ERR_CUDA;
+    return true;
+}
+
+// maps[0] = q, maps[1] = pool rows (gathers), maps[2] = pool pages (boxes)
+inline bool tc_make_maps(const DecodeParams &p, CUtensorMap *maps, bool cached)
+{
+    const uint64_t rows = (uint64_t)p.num_pages * kPage, qrows = (uint64_t)p.batch * p.heads;
+    if (cached)
+        return make_panel_map(&maps[0], p.q, qrows, kTcHeads, kPanels) && make_row_map(&maps[1], p.kv, rows, 1) &&
+               make_panel_map(&maps[2], p.kv, rows, kTile, kPanels);
+    return encode_panel_map(&maps[0], p.q, qrows, kTcHeads, kPanels) && encode_row_map(&maps[1], p.kv, rows, 1, 0) &&
+           encode_panel_map(&maps[2], p.kv, rows, kTile, kPanels);
+}
+
+inline omni_status_t tc_launch(const CUtensorMap *maps, const DecodeParams &p, cudaStream_t stream)
+{
     const int head_groups = (p.heads + kTcHeads - 1) / kTcHeads;
     const unsigned grid = (unsigned)(p.batch * p.splits * head_groups);
     cudaLaunchConfig_t cfg = {};
@@ -815,8 +835,8 @@ inline omni_status_t launch_tc_decode(const DecodeParams &p, cudaStream_t stream
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, tc_decode_kernel, q_map, kv_map, kv_page_map, p) == cudaSuccess ? OMNI_OK
-                                                                                                      : OMNI_ERR_CUDA;
+    return cudaLaunchKernelEx(&cfg, tc_decode_kernel, maps[0], maps[1], maps[2], p) == cudaSuccess ? OMNI_OK
+                                                                                                   : OMNI_ERR_CUDA;
 }
 
 }  // namespace omni

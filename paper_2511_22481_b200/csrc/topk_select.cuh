@@ -75,7 +75,6 @@ topk_select_kernel(const float *__restrict__ scores, const int32_t *__restrict__
     uint32_t crank, nranks;
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(crank));
     asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(nranks));
-    OMNI_SPAN(0);
     // launched with programmatic stream serialization: nothing of the previous kernel in the stream is
     // read or overwritten before this returns
     asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -113,7 +112,6 @@ topk_select_kernel(const float *__restrict__ scores, const int32_t *__restrict__
     int pass = 0;
     for (int shift = 24; shift >= 0; shift -= 8, ++pass) {
         __syncthreads();                                   // keys stored (first pass), histogram copies zeroed
-        if (pass == 0) OMNI_SPAN(1);
         if (few) {
             // few keys are left in the cluster: they go straight into the published histogram
             if (threadIdx.x < 256) sh.published[pass & 1][threadIdx.x] = 0;
@@ -133,7 +131,6 @@ topk_select_kernel(const float *__restrict__ scores, const int32_t *__restrict__
                 if ((key & mask) == prefix) atomicAdd(&sh.replicas[((key >> shift) & 255u) * 32 + lane], 1u);
             }
             __syncthreads();
-            if (pass == 0) OMNI_SPAN(2);
             {
                 // thread t sums half of the 32 copies of bin t / 2 (rotated start keeps the banks apart)
                 const int bin = threadIdx.x >> 1, half = threadIdx.x & 1;
@@ -148,7 +145,6 @@ topk_select_kernel(const float *__restrict__ scores, const int32_t *__restrict__
             for (int i = threadIdx.x; i < 256 * 32; i += kTopkThreads) sh.replicas[i] = 0;
             asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");      // every CTA's histogram is visible
         }
-        if (pass == 0) OMNI_SPAN(3);
         {
             // threads 0..255: bin t of the histogram summed over the cluster, then the bin that holds
             // the need-th largest key: keys in higher bins < need <= keys in this and higher bins
@@ -188,7 +184,6 @@ topk_select_kernel(const float *__restrict__ scores, const int32_t *__restrict__
         need = sh.need;
         few = sh.bin_count <= (uint32_t)kTopkFew;
         mask |= 255u << shift;
-        if (pass == 0) OMNI_SPAN(4);
         // published[] alternates between passes, and the next pass's cluster barrier comes before
         // anybody overwrites the copy read here
         if (need == sh.bin_count) break;                   // every key left under the prefix is taken: the lower digits decide nothing
@@ -197,7 +192,6 @@ topk_select_kernel(const float *__restrict__ scores, const int32_t *__restrict__
     // threshold) tie for the `need` places left, lowest positions first.
     // Warp w owns the contiguous keys [w * per_warp, (w + 1) * per_warp) of the chunk.
     const uint32_t T = prefix | ~mask;                     // largest key under the prefix
-    OMNI_SPAN(5);
     const int per_warp = ((len + kTopkWarps - 1) / kTopkWarps + 127) & ~127;
     const int w_begin = min(len, warp * per_warp), w_end = min(len, w_begin + per_warp);
     uint32_t gt = 0, eq = 0;
@@ -231,7 +225,6 @@ topk_select_kernel(const float *__restrict__ scores, const int32_t *__restrict__
         sh.counts[1] = eq_all;
     }
     topk_cluster_sync();
-    OMNI_SPAN(6);
     // threshold ties and keys above the threshold in the chunks before this one
     {
         uint32_t g[kTopkCluster], e[kTopkCluster];         // all remote loads in flight before the first use
@@ -275,7 +268,6 @@ topk_select_kernel(const float *__restrict__ scores, const int32_t *__restrict__
     }
     if (crank == 0 && threadIdx.x == 0) sel_len[b] = want;
     topk_cluster_sync();                                   // nobody leaves while its counts may still be read
-    OMNI_SPAN(7);
 }
 
 // Launch shape.  A CTA costs about 4 us plus 0.4 us per CTA of its cluster, plus 0.6 us per 1024 keys

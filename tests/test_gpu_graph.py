@@ -2,12 +2,15 @@
 pattern (sparse sink + recent selection on some layers, the full context on the others).  Here a
 few "layers" (each with its own q and its own pattern bit) are captured into one CUDA graph
 through the public entry points and replayed; every layer's result must equal, bit for bit, what
-the same calls produce when launched one by one."""
+the same calls produce when launched one by one, and a sparse and a dense layer of the replay are
+also compared with the CPU oracle."""
+import numpy as np
 import pytest
 import torch
 
 from paper_2511_22481_b200 import binding as B
 from paper_2511_22481_b200 import workloads as W
+from parity import compare, oracle_subset
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
@@ -63,6 +66,18 @@ def test_layer_loop_in_one_cuda_graph_matches_eager():
         assert torch.equal(graph_out[l], eager_out[l]) and torch.equal(graph_lse[l], eager_lse[l]), l
     # the sparse and the dense layers do differ (the pattern is not ignored)
     assert not torch.equal(eager_out[0], eager_out[1])
+    # the replayed results against the oracle: layer 0 on Eq. 2's index set (the workload's own
+    # selection lists are that set), layer 1 on the whole context of every request
+    keep_q = sparse.q
+    sparse.q = qs[0]
+    ref_out, ref_lse, _ = oracle_subset(sparse)
+    compare(graph_out[0].cpu(), graph_lse[0].cpu(), ref_out, ref_lse, "graph replay, compressed layer")
+    dense_idx = torch.arange(max_ctx, dtype=torch.int32, device=DEV).repeat(sparse.batch, 1)
+    keep = (sparse.sel_idx, sparse.sel_len, sparse.max_sel)
+    sparse.q, sparse.sel_idx, sparse.sel_len = qs[1], dense_idx, ctx.clone()
+    ref_out, ref_lse, _ = oracle_subset(sparse)
+    compare(graph_out[1].cpu(), graph_lse[1].cpu(), ref_out, ref_lse, "graph replay, uncompressed layer")
+    sparse.q, (sparse.sel_idx, sparse.sel_len, sparse.max_sel) = keep_q, keep
 
 
 def test_topk_producer_and_decode_in_one_cuda_graph_match_eager():

@@ -155,17 +155,27 @@ def test_rows_outside_the_selection_are_never_used(flags):
         check_workload(w, flags, num_splits=s, what="nan outside S=%d" % s)
 
 
-def test_out_of_range_entries_are_flagged_and_skipped(flags):
+@pytest.mark.parametrize("bad_value", [-3, -2, -1])
+def test_out_of_range_entries_are_flagged_and_skipped(flags, bad_value):
+    # every negative position breaks the contract, -2 included (the kernels use that value
+    # internally as padding of the range form, never on behalf of a caller's list)
     rng = np.random.default_rng(47)
     sel = rng.permutation(8 * 64)[:200].astype(np.int32)
     w = _custom("bad", 47, 128, [8], [sel])
     good = _custom("good", 47, 128, [8], [np.delete(sel, [5, 150])])
     bad_idx = w.sel_idx.clone()
-    bad_idx[0, 5] = -3
+    bad_idx[0, 5] = bad_value
     bad_idx[0, 150] = 8 * 64 + 1
     w.sel_idx = bad_idx
     plan = run_gpu(w, flags)
     assert int(plan.status.item()) & B.OMNI_DEV_BAD_INDEX
+    # a lone -2 must be flagged by the decode kernel as well, not only next to another bad entry
+    only = w.sel_idx.clone()
+    only[0, 150] = sel[150]
+    w.sel_idx = only
+    plan1 = run_gpu(w, flags)
+    assert int(plan1.status.item()) & B.OMNI_DEV_BAD_INDEX
+    w.sel_idx = bad_idx
     ref_out, ref_lse, _ = oracle_subset(good)
     compare(plan.out.cpu(), plan.lse.cpu(), ref_out, ref_lse, "skip bad entries")
     desc = B.make_desc(1, 128, w.num_pages, w.max_pages_per_req, w.max_sel, w.scale)
@@ -321,11 +331,12 @@ def test_host_buffer_entry_point_two_halves(flags, batch):
     compare(out_h, lse_h, ref_out, ref_lse, "host entry point, two halves")
 
 
-# ------------------------------------------------------------------ full benchmark sizes, sampled
+# ------------------------------------------------------------------ full benchmark sizes
 
-def test_config2_full_size_sampled(flags):
+def test_config2_full_size_every_row(flags):
+    """Config 2 in the launch configuration the benchmark times: every (request, head) row."""
     w = W.config2_r1(DEV)
-    check_workload(w, flags, reqs=[0, 13, 31], heads=[0, 63, 64, 127], what="config2", strict_abs=True)
+    check_workload(w, flags, what="config2", strict_abs=True)
 
 
 def test_config2_2048_variant(flags):
@@ -333,21 +344,39 @@ def test_config2_2048_variant(flags):
     check_workload(w, flags, reqs=[7], heads=[1, 100], what="config2/2048", strict_abs=True)
 
 
-def test_config3_ragged_full_size_sampled(flags):
+def test_config3_ragged_full_size_sixteen_requests_all_heads(flags):
     w = W.config3_ragged(DEV)
     sl = w.sel_len.cpu().numpy()
-    reqs = sorted({int(sl.argmin()), int(sl.argmax()), 0, 127})
-    check_workload(w, flags, reqs=reqs, heads=[0, 77, 127], what="config3", strict_abs=True)
+    order = np.argsort(sl, kind="stable")
+    # the shortest and the longest selections, the first and the last request, and a spread of the rest
+    reqs = sorted({int(order[0]), int(order[1]), int(order[-1]), int(order[-2]), 0, 127} |
+                  {int(order[i]) for i in range(5, 128, 12)})
+    assert len(reqs) >= 16
+    check_workload(w, flags, reqs=reqs, what="config3", strict_abs=True)
 
 
-def test_config4_topk_full_size_sampled(flags):
+def test_config4_topk_full_size_every_row(flags):
     w = W.config4_topk(DEV)
-    check_workload(w, flags, reqs=[0, 15], heads=[0, 64, 127], what="config4", strict_abs=True)
+    check_workload(w, flags, what="config4", strict_abs=True)
 
 
-def test_config5_cells_sampled():
-    for batch, n in ((1, 512), (8, 8192), (32, 2048)):
-        w = W.config5_cell(batch, n, DEV)
-        check_workload(w, 0, reqs=[batch - 1], heads=[5, 126], what="config5 B%d N%d" % (batch, n), strict_abs=True)
-    w = W.config5_cell(1, 512, DEV, dense_variant=True)
-    check_workload(w, 0, reqs=[0], heads=[9], what="config5 dense B1", strict_abs=True)
+def _sample_requests(batch):
+    """First, last and two interior requests (at most four): with more work units than the device
+    runs at once, these sit in different waves of the launch."""
+    return sorted({0, batch // 3, (2 * batch) // 3, batch - 1})
+
+
+@pytest.mark.parametrize("batch,n", [(1, 512), (8, 8192), (32, 2048), (32, 8192), (128, 512), (128, 8192),
+                                     (256, 2048), (256, 8192)])
+def test_config5_sparse_cells_sampled_all_heads(batch, n):
+    w = W.config5_cell(batch, n, DEV)
+    check_workload(w, 0, reqs=_sample_requests(batch), what="config5 B%d N%d" % (batch, n), strict_abs=True)
+
+
+@pytest.mark.parametrize("batch", [1, 8, 32])
+def test_config5_dense_cells_sampled_all_heads(batch):
+    """The dense arm of the sweep (all 65536 tokens): several splits per request and a separate
+    merge launch from batch 8 on."""
+    w = W.config5_cell(batch, 2048, DEV, dense_variant=True)
+    reqs = _sample_requests(batch)[:2] if batch > 1 else [0]
+    check_workload(w, 0, reqs=reqs, what="config5 dense B%d" % batch, strict_abs=True)

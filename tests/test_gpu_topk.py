@@ -73,6 +73,20 @@ def test_special_values():
     _check(scores, [stride, stride, stride], stride)
 
 
+def test_nans_with_mixed_sign_bits_rank_by_position():
+    """k reaches into the NaNs, which carry either sign bit: all NaNs are equal, lowest positions win."""
+    rng = np.random.default_rng(8)
+    stride, k = 5000, 3000
+    scores = rng.standard_normal((2, stride)).astype(np.float32)
+    bits = scores.view(np.uint32)
+    nan_at = rng.random((2, stride)) < 0.6
+    neg = rng.random((2, stride)) < 0.5
+    bits[nan_at & neg] = 0xFFC00000
+    bits[nan_at & ~neg] = 0x7FC00001
+    assert np.isnan(scores[nan_at]).all()
+    _check(scores, [stride, 4321], k)
+
+
 def test_keys_that_differ_only_in_low_bits():
     base = np.float32(1.0).view(np.uint32)
     rng = np.random.default_rng(6)

@@ -19,6 +19,18 @@ def test_hand_worked_ties_take_the_lowest_positions():
     assert topk_positions(s, 0, 2).tolist() == []
 
 
+def test_nans_of_either_sign_are_equal_and_ordered_by_position():
+    neg_nan = np.array([0xFFC00000], dtype=np.uint32).view(np.float32)[0]      # NaN with the sign bit set
+    pos_nan = np.float32(np.nan)
+    assert np.signbit(neg_nan) and np.isnan(neg_nan) and not np.signbit(pos_nan)
+    s = np.array([neg_nan, 1.0, pos_nan, neg_nan, pos_nan], dtype=np.float32)
+    # one number, then the NaNs in order of position, whatever their sign bits
+    assert topk_positions(s, 5, 1).tolist() == [1]
+    assert topk_positions(s, 5, 2).tolist() == [0, 1]
+    assert topk_positions(s, 5, 3).tolist() == [0, 1, 2]
+    assert topk_positions(s, 5, 4).tolist() == [0, 1, 2, 3]
+
+
 def test_hand_worked_zero_signs_nan_and_infinities():
     s = np.array([0.0, -0.0, np.nan, -1.0, np.inf, -np.inf], dtype=np.float32)
     assert topk_positions(s, 6, 1).tolist() == [4]

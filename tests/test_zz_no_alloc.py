@@ -6,8 +6,8 @@ cannot afford the device-wide synchronisation an allocation implies.  For them
 ``omni_sparse_mla_decode_static`` keeps the split-KV scratch in a fixed array inside the library.
 These tests call it through the C ABI twice in a row (the array keeps the first call's
 contents, so the second call shows that stale scratch does no harm) and compare each result
-with ``omni_sparse_mla_decode`` on the same inputs, under the same tolerance as the other
-parity tests.  The file name sorts last so that a run that stops at the first failure has
+with ``omni_sparse_mla_decode`` on the same inputs and with the CPU oracle, under the same
+tolerance as the other parity tests.  The file name sorts last so that a run that stops at the first failure has
 already run every other test.
 """
 import ctypes
@@ -19,7 +19,7 @@ import torch
 from paper_2511_22481_b200 import binding as B
 from paper_2511_22481_b200 import build as builder
 from paper_2511_22481_b200 import workloads as W
-from parity import ABS_TOL, LSE_TOL
+from parity import ABS_TOL, LSE_TOL, compare, oracle_subset
 
 
 def _desc(w, num_splits=0):
@@ -65,6 +65,8 @@ def test_static_scratch_decode_matches_workspace_decode_twice_in_a_row():
         torch.cuda.synchronize()
         out, lse = _static(w, desc)
         _same(out, lse, plan.out, plan.lse)
+        ref_out, ref_lse, _ = oracle_subset(w)
+        compare(out.cpu(), lse.cpu(), ref_out, ref_lse, "static scratch entry point, splits=%d" % splits)
 
 
 @pytest.mark.gpu
