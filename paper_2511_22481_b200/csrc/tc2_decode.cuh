@@ -27,8 +27,8 @@
 // Warps per CTA: 0 K-role producer, 1 MMA issuer (CTA 0 only) + tensor-memory owner,
 // 2-5 and 8-11 softmax / epilogue (two warps per tensor-memory lane quarter, 16 of a tile's 64
 // tokens per thread), 6 V-role producer, 7 L2 prefetcher (CTA 0 only): shared memory holds
-// only two tiles, about one HBM latency of work, so whole pages are pulled into L2 a few tiles
-// ahead and the shared-memory refills then hit L2.
+// only two tiles, about one HBM latency of work, so each whole page is pulled into L2 one tile
+// before its K-role load and the shared-memory refills start from a line already on its way.
 //
 // Tensor memory per CTA (a 64-row slice of an M=128 pair accumulator keeps columns [0, N/2) in
 // lanes 0-63 and columns [N/2, N) in lanes 64-127):
@@ -51,7 +51,10 @@ namespace omni {
 
 constexpr int kC2Tile = 64;                              // tokens per tile of the pair
 constexpr int kC2Threads = 384;
-constexpr int kPrefetchAhead = 5;                         // tiles the L2 prefetch runs ahead of Q K^T
+// Tiles the L2 prefetch runs ahead of the K-role loads.  Measured on B200: the further ahead, the
+// slower (1: 30.4 us, 5: 32.3 us, 12: 35.0 us per step on the batch-32 benchmark shape; the same
+// order at batch 128): a line prefetched long before its use is often gone again by then.
+constexpr int kPrefetchAhead = 1;
 constexpr int kC2KBytes = kPanels * 32 * 128;            // K role: 9 panels x [32 tokens x 128 B]
 constexpr int kC2KPanel = 32 * 128;
 constexpr int kC2VBytes = 4 * kPanelBytes;               // V role: 4 panels x [64 tokens x 128 B]
@@ -63,7 +66,11 @@ constexpr int kC2SmemCtl = kC2SmemP + 2 * kPanelBytes;
 constexpr int kC2SmemCtlBytes = 3072;
 constexpr int kC2SmemBytes = kC2SmemCtl + kC2SmemCtlBytes;   // no alignment slack: the base is checked at run time
 constexpr uint32_t kC2ColS = 256;
-constexpr int kMaskRing = 4;
+// Validity masks travel from the K producer to the softmax warps through a small ring.  The
+// producer writes the mask of tile i+1 once the score MMAs of tile i-2 have retired, and those
+// were issued only after every softmax warp had read the scores of tile i-5 (three score
+// buffers), i.e. after tile i-6 was finished: seven tiles can be live, so the ring holds eight.
+constexpr int kMaskRing = 8;
 
 struct C2Control {
     uint64_t q_full;
@@ -561,16 +568,22 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
             stage_pages(x1);
             stage_rows(0, x0, row_lo, row_hi, mask, contig, contig_lo, contig_hi, any_bad);
         }
+        // The mask of a tile is published (store + fence) right after its rows are resolved and
+        // BEFORE the next index loads go out: a fence waits for the loads its thread has in
+        // flight, so a fence placed after them put their whole latency in front of every refill.
+        auto publish_mask = [&](int tile) {
+            if (lane == 0) {
+                ctl->valid_mask[tile % kMaskRing] = mask;
+                __threadfence_block();
+            }
+        };
+        publish_mask(0);
         bool ok = true;
         int pending = -1;                    // stage of a gathered tile whose bytes are not credited yet
         const char *kv_bytes = reinterpret_cast<const char *>(p.kv);
         for (int i = 0; ok && i < tiles; ++i) {
             const int st = i & 1;
-            if (lane == 0) {
-                *const_cast<volatile int32_t *>(&ctl->k_progress) = i;
-                ctl->valid_mask[i % kMaskRing] = mask;
-                __threadfence_block();
-            }
+            if (lane == 0) *const_cast<volatile int32_t *>(&ctl->k_progress) = i;
             if (i >= 2) ok = mbar_wait(&ctl->k_empty[st], ((i >> 1) - 1) & 1);
             ok = __all_sync(0xffffffffu, ok) && (*abort_flag == 0);
             if (!ok) break;
@@ -594,7 +607,10 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
             }
             if (gathered) pending = st;
             // advance the index pipeline: rows of tile i+1, page ids of tile i+2, positions of tile i+3
-            if (i + 1 < tiles) stage_rows(i + 1, x1, row_lo, row_hi, mask, contig, contig_lo, contig_hi, any_bad);
+            if (i + 1 < tiles) {
+                stage_rows(i + 1, x1, row_lo, row_hi, mask, contig, contig_lo, contig_hi, any_bad);
+                publish_mask(i + 1);
+            }
             x1 = x2;
             stage_pages(x1);
             stage_tokens(i + 3, x2);
