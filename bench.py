@@ -152,7 +152,15 @@ def _oracle_sample(w, target_s=15.0, max_requests=None):
         total_t += t
         total_tok += tokens
         passes += 1
-    return dict(seconds=total_t, tokens=total_tok, requests=n, passes=passes, cores=oracle.num_threads())
+    # the float build of the same source, one pass over the same requests (a second CPU figure)
+    reqs = slice(0, n)
+    pt, si, sl = w.page_table[reqs].cpu().numpy(), w.sel_idx[reqs].cpu().numpy(), w.sel_len[reqs].cpu().numpy()
+    rows = oracle.resolve_rows(pt, si, sl, w.page_size, w.num_pages)
+    gather = torch.from_numpy(np.where(rows < 0, 0, rows)).to(w.kv_cache.device)
+    krows = w.kv_cache.view(-1, w.d_qk)[gather.view(-1)].view(rows.shape[0], -1, w.d_qk).cpu()
+    f32_seconds, _, _ = oracle.attend_rows_f32_timed(w.q[reqs].cpu(), krows, sl, w.d_v, w.scale)
+    return dict(seconds=total_t, tokens=total_tok, requests=n, passes=passes, cores=oracle.num_threads(),
+                f32_seconds=f32_seconds, f32_tokens=int(sl.sum()))
 
 
 WORKLOAD_HELP = ("config2 (default, the named benchmark) | config1 | config3 | config4 | "
@@ -523,7 +531,10 @@ def main():
                 "sample": "fp64 oracle on the first %d of %d requests, all 128 heads, %d passes (%d selected tokens in all), "
                           "%.1f s; one full step extrapolates to %.0f us"
                           % (s["requests"], w.batch, s["passes"], s["tokens"], s["seconds"],
-                             s["seconds"] / s["tokens"] * w.selected_tokens * 1e6)}
+                             s["seconds"] / s["tokens"] * w.selected_tokens * 1e6),
+                "fp32_build": {"value": round(s["f32_tokens"] * KV_ROW_BYTES / s["f32_seconds"] / 1e9, 5), "unit": "GB/s",
+                               "note": "the same oracle source compiled with float as its working type, one pass over "
+                                       "the same requests; timed only, never a reference"}}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

@@ -36,6 +36,45 @@ def build(force: bool = False) -> str:
     return _LIB
 
 
+_LIB32 = os.path.join(_HERE, "libsparse_mla_oracle_f32.so")
+_lib32 = None
+
+
+def build_f32(force: bool = False) -> str:
+    """The same source compiled with float as its working type.  Timed by the benchmark as the
+    plain fp32 CPU figure; never a reference for anything."""
+    with _lock:
+        stale = (not os.path.exists(_LIB32)) or os.path.getmtime(_LIB32) < os.path.getmtime(_SRC)
+        if force or stale:
+            tmp = _LIB32 + ".tmp.%d" % os.getpid()
+            cmd = ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11", "-DORACLE_REAL=float", "-o", tmp, _SRC, "-lm"]
+            subprocess.run(cmd, check=True)
+            os.replace(tmp, _LIB32)
+    return _LIB32
+
+
+def attend_rows_f32_timed(q, krows, n, d_v: int, scale: float):
+    """Runs the float build of oracle_attend_rows on the same arguments as ``attend_rows``
+    and returns (seconds, out, lse); for timing only."""
+    import time
+    global _lib32
+    if _lib32 is None:
+        build_f32()
+        lib = ctypes.CDLL(_LIB32)
+        i32, f64, vp = ctypes.c_int, ctypes.c_double, ctypes.c_void_p
+        lib.oracle_attend_rows.argtypes = [i32, i32, i32, i32, i32, f64, vp, vp, vp, vp, vp, vp]
+        lib.oracle_attend_rows.restype = None
+        _lib32 = lib
+    qb, kb, nn = bf16_bits(q), bf16_bits(krows), _i32(n)
+    B, H, d_qk = qb.shape
+    max_sel = kb.shape[1]
+    out = np.empty((B, H, d_v), dtype=np.float64)
+    lse = np.empty((B, H), dtype=np.float64)
+    t0 = time.perf_counter()
+    _lib32.oracle_attend_rows(B, H, d_qk, d_v, max_sel, float(scale), _p(qb), _p(kb), _p(nn), _p(out), _p(lse), None)
+    return time.perf_counter() - t0, out, lse
+
+
 def _load():
     global _lib
     if _lib is None:

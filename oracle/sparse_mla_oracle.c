@@ -17,6 +17,10 @@
  *
  * Everything is two-pass fp64: scores, then max, then exp/sum, then the weighted sum.
  * No tiling, no online recurrence, no fusion.  bf16 inputs are widened exactly.
+ * The working type of oracle_attend_rows is the typedef `real` (double unless the file is
+ * compiled with -DORACLE_REAL=float): the fp64 build is the oracle every test compares with;
+ * the float build of the same source exists only to be timed as the "plain fp32 CPU" figure
+ * of the benchmark and is never used as a reference.
  *
  * Parity status of each exported function (pins live in tests/test_oracle_pins.py):
  *   oracle_resolve_rows      pinned (hand-written tables, histogram/spike constructions)
@@ -33,6 +37,11 @@
 #ifdef _OPENMP
 #include <omp.h>
 #endif
+
+#ifndef ORACLE_REAL
+#define ORACLE_REAL double
+#endif
+typedef ORACLE_REAL real;
 
 /* bf16 bit pattern -> double, exact (bf16 is the top half of an IEEE-754 binary32). */
 static double bf16_to_double(uint16_t bits)
@@ -99,55 +108,61 @@ void oracle_attend_rows(int batch, int heads, int d_qk, int d_v, int max_sel, do
     const long total = (long)batch * heads;
 #pragma omp parallel
     {
-        double *x = (double *)malloc(sizeof(double) * (size_t)(max_sel > 0 ? max_sel : 1));
-        double *qd = (double *)malloc(sizeof(double) * (size_t)d_qk);
+        real *x = (real *)malloc(sizeof(real) * (size_t)(max_sel > 0 ? max_sel : 1));
+        real *qd = (real *)malloc(sizeof(real) * (size_t)d_qk);
+        real *oa = (real *)malloc(sizeof(real) * (size_t)(d_v > 0 ? d_v : 1));
 #pragma omp for schedule(dynamic, 1)
         for (long bh = 0; bh < total; ++bh) {
             const int b = (int)(bh / heads);
             const int nb = n[b];
             double *o = out + (size_t)bh * d_v;
             for (int d = 0; d < d_v; ++d)
-                o[d] = 0.0;
+                oa[d] = (real)0.0;
             if (nb <= 0) {
+                for (int d = 0; d < d_v; ++d)
+                    o[d] = 0.0;
                 lse[bh] = -INFINITY;
                 if (wsum)
                     wsum[bh] = 0.0;
                 continue;
             }
             for (int c = 0; c < d_qk; ++c)
-                qd[c] = bf16_to_double(q[(size_t)bh * d_qk + c]);
+                qd[c] = (real)bf16_to_double(q[(size_t)bh * d_qk + c]);
             const uint16_t *kb = krows + (size_t)b * max_sel * d_qk;
             /* pass 1: scaled scores x_j = scale * <q, k_j> */
             for (int j = 0; j < nb; ++j) {
                 const uint16_t *k = kb + (size_t)j * d_qk;
-                double acc = 0.0;
+                real acc = (real)0.0;
                 for (int c = 0; c < d_qk; ++c)
-                    acc += qd[c] * bf16_to_double(k[c]);
-                x[j] = scale * acc;
+                    acc += qd[c] * (real)bf16_to_double(k[c]);
+                x[j] = (real)scale * acc;
             }
             /* pass 2: max, partition function */
-            double m = x[0];
+            real m = x[0];
             for (int j = 1; j < nb; ++j)
                 if (x[j] > m)
                     m = x[j];
-            double z = 0.0;
+            real z = (real)0.0;
             for (int j = 0; j < nb; ++j)
-                z += exp(x[j] - m);
-            lse[bh] = m + log(z);
+                z += (real)exp((double)(x[j] - m));
+            lse[bh] = (double)(m + (real)log((double)z));
             /* pass 3: weighted sum of the value part of each row */
-            double ws = 0.0;
+            real ws = (real)0.0;
             for (int j = 0; j < nb; ++j) {
-                const double w = exp(x[j] - m) / z;
+                const real w = (real)exp((double)(x[j] - m)) / z;
                 ws += w;
                 const uint16_t *v = kb + (size_t)j * d_qk;
                 for (int d = 0; d < d_v; ++d)
-                    o[d] += w * bf16_to_double(v[d]);
+                    oa[d] += w * (real)bf16_to_double(v[d]);
             }
+            for (int d = 0; d < d_v; ++d)
+                o[d] = (double)oa[d];
             if (wsum)
-                wsum[bh] = ws;
+                wsum[bh] = (double)ws;
         }
         free(x);
         free(qd);
+        free(oa);
     }
 }
 
