@@ -290,6 +290,20 @@ omni_status_t omni_sparse_mla_combine(const omni_mla_desc_t *desc, int32_t max_s
                                       void *stream);
 
 /*
+ * Self-test of the bounded device waits (no counterpart in the paper).  Every wait inside the
+ * kernels of this library (on a copy, on the tensor core, on another warp or CTA) gives up
+ * after a limit, ORs OMNI_DEV_TIMEOUT plus a role bit into *device_status and lets the kernel
+ * return; nothing spins without bound and nothing traps.  This entry point exercises exactly
+ * that helper where it can be made to run out on purpose without involving a copy or tensor
+ * memory: one warp waits for `limit_cycles` SM clocks (1 .. 2^31) on a barrier nobody arrives
+ * on.  Afterwards *device_status carries OMNI_DEV_TIMEOUT and, if waited_cycles is non-NULL
+ * (device pointer, 8-byte aligned), *waited_cycles the clocks the wait took.  The context
+ * stays usable.  Asynchronous on `stream`.
+ */
+omni_status_t omni_selftest_bounded_wait(int64_t limit_cycles, int32_t *device_status,
+                                         int64_t *waited_cycles, void *stream);
+
+/*
  * Index contract check on the device: ORs OMNI_DEV_BAD_INDEX into *device_status if any
  * sel_len[b] lies outside [0, max_sel], any read position is negative or beyond the page
  * table row, or any page id it reaches lies outside [0, num_pages).  Launches one small

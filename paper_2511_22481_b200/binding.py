@@ -34,6 +34,7 @@ EXPORTS = (
     "omni_sparse_mla_host_staging_bytes", "omni_sparse_mla_decode_host",
     "omni_sparse_mla_set_profile_events", "omni_sparse_mla_decode_static",
     "omni_sparse_mla_plan_init", "omni_sparse_mla_decode_planned", "omni_sparse_mla_plan_query",
+    "omni_selftest_bounded_wait",
 )
 
 
@@ -107,6 +108,8 @@ def load() -> ctypes.CDLL:
     lib.omni_sparse_mla_decode_host.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp, sz, vp, vp]
     lib.omni_sparse_mla_decode_static.restype = ctypes.c_int
     lib.omni_sparse_mla_decode_static.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.omni_selftest_bounded_wait.restype = ctypes.c_int
+    lib.omni_selftest_bounded_wait.argtypes = [ctypes.c_int64, vp, vp, vp]
     lib.omni_sparse_mla_plan_query.restype = i32
     lib.omni_sparse_mla_plan_query.argtypes = [dp, i32, i32, ctypes.POINTER(ctypes.c_int32)]
     lib.omni_sparse_mla_plan_init.restype = ctypes.c_int
@@ -339,6 +342,14 @@ def omni_sparse_mla_combine(desc, max_splits, part_out, part_lse, num_splits, ou
         _ptr(out, torch.bfloat16, "cuda", "out"), _ptr(lse, torch.float32, "cuda", "lse"),
         _stream(stream))
     _check(code, "omni_sparse_mla_combine")
+
+
+def omni_selftest_bounded_wait(limit_cycles, device_status, waited_cycles=None, stream=None) -> None:
+    """One warp waits `limit_cycles` SM clocks on a barrier nobody arrives on, then reports the time-out."""
+    code = load().omni_selftest_bounded_wait(
+        int(limit_cycles), _ptr(device_status, torch.int32, "cuda", "device_status"),
+        _ptr(waited_cycles, torch.int64, "cuda", "waited_cycles"), _stream(stream))
+    _check(code, "omni_selftest_bounded_wait")
 
 
 def omni_sparse_mla_validate(desc, page_table, sel_idx, sel_len, device_status, stream=None) -> None:

@@ -193,6 +193,28 @@ omni_status_t launch_resolve(const omni_mla_desc_t *d, const int32_t *page_table
     return cudaPeekAtLastError() == cudaSuccess ? OMNI_OK : OMNI_ERR_CUDA;
 }
 
+// Self-test of the bounded wait every kernel here relies on: one warp waits, with the given
+// limit, on a barrier that nobody ever arrives on.  No copy and no tensor memory is involved;
+// the warp reports what the product kernels report when a wait runs out and returns.
+__global__ void __launch_bounds__(32) bounded_wait_selftest_kernel(long long limit_cycles, int32_t *status,
+                                                                   long long *waited_cycles)
+{
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    const long long t0 = clock64();
+    bool ok = mbar_wait(&bar, 0, limit_cycles);
+    ok = __all_sync(0xffffffffu, ok);
+    const long long t1 = clock64();
+    if (threadIdx.x == 0) {
+        if (!ok) flag_status(status, OMNI_DEV_TIMEOUT | OMNI_DEV_ROLE_SOFTMAX);
+        if (waited_cycles) *waited_cycles = t1 - t0;
+    }
+}
+
 }  // namespace
 }  // namespace omni
 
@@ -545,6 +567,17 @@ omni_status_t omni_sparse_mla_combine(const omni_mla_desc_t *desc, int32_t max_s
         return OMNI_ERR_ALIGN;
     return launch_combine(desc->batch, desc->num_heads, max_splits, part_out, part_lse, num_splits,
                           out, lse, static_cast<cudaStream_t>(stream));
+}
+
+omni_status_t omni_selftest_bounded_wait(int64_t limit_cycles, int32_t *device_status, int64_t *waited_cycles,
+                                         void *stream)
+{
+    if (!device_status) return OMNI_ERR_NULL;
+    if (limit_cycles < 1 || limit_cycles > ((int64_t)1 << 31)) return OMNI_ERR_SHAPE;
+    if (!aligned(device_status, 4) || !aligned(waited_cycles, 8)) return OMNI_ERR_ALIGN;
+    bounded_wait_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(
+        (long long)limit_cycles, device_status, reinterpret_cast<long long *>(waited_cycles));
+    return cudaPeekAtLastError() == cudaSuccess ? OMNI_OK : OMNI_ERR_CUDA;
 }
 
 omni_status_t omni_sparse_mla_validate(const omni_mla_desc_t *desc, const int32_t *page_table,

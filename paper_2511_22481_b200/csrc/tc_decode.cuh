@@ -88,8 +88,9 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes)
                  : "memory");
 }
 
-// Bounded wait on a phase parity; false if about a second passed without the phase completing.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity)
+// Bounded wait on a phase parity; false if `limit` SM clocks (about a second by default) passed
+// without the phase completing.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, long long limit = kWaitCycles)
 {
     const uint32_t addr = smem_u32(bar);
     const long long start = clock64();
@@ -103,7 +104,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity)
             : "r"(addr), "r"(parity)
             : "memory");
         if (done) return true;
-        if ((it & 63u) == 63u && clock64() - start > kWaitCycles) return false;
+        if ((it & 63u) == 63u && clock64() - start > limit) return false;
     }
 }
 
