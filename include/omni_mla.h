@@ -247,6 +247,39 @@ omni_status_t omni_sparse_mla_decode_rolling(const omni_mla_desc_t *desc, const 
                                              size_t workspace_bytes, int32_t *device_status, void *stream);
 
 /*
+ * 8-bit latent cache (the paper serves an INT8-quantised model, Evaluation, "Experimental
+ * Setup", and gives no cache format; this one is the library's own).  A token's row is
+ * OMNI_Q8_ROW_BYTES = 640 bytes: its 512 latent columns as FP8 E4M3 codes (1-4-3 bits, bias 7,
+ * largest magnitude 448, no infinities), then its 64 rope columns unchanged as bf16.  One fp32
+ * scale per row lives in a second array; a latent value is code * scale.
+ *
+ * omni_kv_quantize_q8 writes that form for `num_rows` bf16 rows (kv_rows bf16 [num_rows, 576],
+ * 16-byte aligned; kv_q8 uint8 [num_rows, 640], 128-byte aligned; kv_scale fp32 [num_rows]):
+ *     scale = max(amax, 2^-60) / 448,  amax = largest |value| of the row's 512 latent columns
+ *     code  = E4M3(value / scale)      fp32 division, round to nearest even, saturating at 448
+ * Rows map one to one, so a paged pool keeps its page table.
+ *
+ * omni_sparse_mla_decode_q8 is omni_sparse_mla_decode over such a pool (kv_q8 uint8
+ * [num_pages, 64, 640], kv_scale fp32 [num_pages, 64]): the result is DEFINED as Eq. 1's
+ * restricted attention over the de-quantised rows (code * scale for the latent columns, the
+ * stored bf16 for the rope columns), K = all 576 columns, V = the first 512.  The codes go
+ * through the 8-bit tensor-core path unchanged; q and the softmax weights enter it as two
+ * E4M3 terms each (value ~ hi + lo), which keeps about the eight significant bits they have in
+ * the bf16 path, so the same tolerances apply against that definition.  Needs more than 64
+ * heads (OMNI_ERR_SHAPE otherwise, and for OMNI_FLAG_SIMT); descriptor, index arrays,
+ * workspace (omni_sparse_mla_workspace_bytes), status word, stream and the remaining flags are
+ * those of omni_sparse_mla_decode.  Rows that are not selected are never read, scales included.
+ */
+#define OMNI_Q8_ROW_BYTES 640
+omni_status_t omni_kv_quantize_q8(const void *kv_rows, int64_t num_rows, void *kv_q8, float *kv_scale,
+                                  void *stream);
+omni_status_t omni_sparse_mla_decode_q8(const omni_mla_desc_t *desc, const void *q, const void *kv_q8,
+                                        const float *kv_scale, const int32_t *page_table,
+                                        const int32_t *sel_idx, const int32_t *sel_len, void *out,
+                                        float *lse, void *workspace, size_t workspace_bytes,
+                                        int32_t *device_status, void *stream);
+
+/*
  * Selection producer for token-level sparsity (the step before the decode call when the index
  * set is "the k highest-scoring tokens", as in a top-k sparse attention variant; the paper
  * itself only uses the sink + recent rule of Eq. 2).  For every request b with M = ctx_len[b]

@@ -9,9 +9,10 @@ checked against it:
     FP8 E4M3 codes (1 sign, 4 exponent bits with bias 7, 3 mantissa bits; no infinities; the
     largest finite magnitude is 448; exponent field 0 holds subnormals m/8 * 2^-6), followed by
     the 64 rope columns unchanged as bf16 (128 bytes);
-  * one fp32 scale per row, kept in a separate array: scale = amax / 448 with amax the largest
-    |value| of the row's 512 latent columns (scale = 1 when amax = 0); code = E4M3(value / scale),
-    the division done in fp32 and the result rounded to nearest, ties to even, saturating at 448;
+  * one fp32 scale per row, kept in a separate array: scale = max(amax, 2^-60) / 448 with amax
+    the largest |value| of the row's 512 latent columns (the floor keeps the scale and its
+    reciprocal finite for all-zero rows); code = E4M3(value / scale), both divisions done in fp32,
+    the result rounded to nearest, ties to even, saturating at 448;
   * the value a code stands for is exactly decode(code) * scale (an fp32 product, taken exactly
     here in fp64), and the result of the 8-bit decode call is DEFINED as Eq. 1's restricted
     attention over those exactly de-quantised rows (rope columns as stored), with K = all 576
@@ -83,7 +84,7 @@ def quantise_rows(row_bits):
     assert bits.ndim == 2 and bits.shape[1] == NOPE + ROPE
     x = _bf16_bits_to_f32(bits[:, :NOPE])
     amax = np.abs(x).max(axis=1).astype(np.float32)
-    scale = np.where(amax > 0, amax / np.float32(E4M3_MAX), np.float32(1.0)).astype(np.float32)
+    scale = (np.maximum(amax, np.float32(2.0 ** -60)) / np.float32(E4M3_MAX)).astype(np.float32)
     codes = e4m3_encode((x / scale[:, None]).astype(np.float32))
     out = np.empty((bits.shape[0], ROW_BYTES), dtype=np.uint8)
     out[:, :NOPE] = codes

@@ -34,7 +34,7 @@ EXPORTS = (
     "omni_sparse_mla_host_staging_bytes", "omni_sparse_mla_decode_host",
     "omni_sparse_mla_set_profile_events", "omni_sparse_mla_decode_static",
     "omni_sparse_mla_plan_init", "omni_sparse_mla_decode_planned", "omni_sparse_mla_plan_query",
-    "omni_selftest_bounded_wait",
+    "omni_selftest_bounded_wait", "omni_kv_quantize_q8", "omni_sparse_mla_decode_q8",
 )
 
 
@@ -108,6 +108,10 @@ def load() -> ctypes.CDLL:
     lib.omni_sparse_mla_decode_host.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp, sz, vp, vp]
     lib.omni_sparse_mla_decode_static.restype = ctypes.c_int
     lib.omni_sparse_mla_decode_static.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.omni_kv_quantize_q8.restype = ctypes.c_int
+    lib.omni_kv_quantize_q8.argtypes = [vp, ctypes.c_int64, vp, vp, vp]
+    lib.omni_sparse_mla_decode_q8.restype = ctypes.c_int
+    lib.omni_sparse_mla_decode_q8.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
     lib.omni_selftest_bounded_wait.restype = ctypes.c_int
     lib.omni_selftest_bounded_wait.argtypes = [ctypes.c_int64, vp, vp, vp]
     lib.omni_sparse_mla_plan_query.restype = i32
@@ -258,6 +262,32 @@ def omni_sparse_mla_decode_rolling(desc, q, kv_cache, page_table, ctx_len, n_sin
         None if workspace is None else ctypes.c_void_p(workspace.data_ptr()), ws_bytes,
         _ptr(device_status, torch.int32, "cuda", "device_status"), _stream(stream))
     _check(code, "omni_sparse_mla_decode_rolling")
+
+
+OMNI_Q8_ROW_BYTES = 640
+
+
+def omni_kv_quantize_q8(kv_rows, kv_q8, kv_scale, stream=None) -> None:
+    """bf16 rows [..., 576] -> 8-bit cache rows [..., 640] (uint8) and one fp32 scale per row."""
+    num_rows = kv_rows.numel() // 576
+    code = load().omni_kv_quantize_q8(
+        _ptr(kv_rows, torch.bfloat16, "cuda", "kv_rows"), int(num_rows), _ptr(kv_q8, torch.uint8, "cuda", "kv_q8"),
+        _ptr(kv_scale, torch.float32, "cuda", "kv_scale"), _stream(stream))
+    _check(code, "omni_kv_quantize_q8")
+
+
+def omni_sparse_mla_decode_q8(desc, q, kv_q8, kv_scale, page_table, sel_idx, sel_len, out, lse,
+                              workspace=None, device_status=None, stream=None) -> None:
+    """Decode over the 8-bit latent cache (see ``omni_kv_quantize_q8``)."""
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    code = load().omni_sparse_mla_decode_q8(
+        ctypes.byref(desc), _ptr(q, torch.bfloat16, "cuda", "q"), _ptr(kv_q8, torch.uint8, "cuda", "kv_q8"),
+        _ptr(kv_scale, torch.float32, "cuda", "kv_scale"), _ptr(page_table, torch.int32, "cuda", "page_table"),
+        _ptr(sel_idx, torch.int32, "cuda", "sel_idx"), _ptr(sel_len, torch.int32, "cuda", "sel_len"),
+        _ptr(out, torch.bfloat16, "cuda", "out"), _ptr(lse, torch.float32, "cuda", "lse"),
+        None if workspace is None else ctypes.c_void_p(workspace.data_ptr()), ws_bytes,
+        _ptr(device_status, torch.int32, "cuda", "device_status"), _stream(stream))
+    _check(code, "omni_sparse_mla_decode_q8")
 
 
 OMNI_PLAN_BYTES = 1024

@@ -9,6 +9,7 @@
 #include "simt_decode.cuh"
 #include "tc_decode.cuh"
 #include "tc2_decode.cuh"
+#include "tc2q8_decode.cuh"
 #include "topk_select.cuh"
 
 namespace omni {
@@ -289,32 +290,36 @@ size_t omni_sparse_mla_workspace_bytes(const omni_mla_desc_t *desc)
 constexpr uint32_t kPlanMagic = 0x4c504d4fu;
 struct LaunchPlan {
     uint32_t magic;
-    int32_t kernel;            // 0 plain-FMA, 1 single-CTA tensor-core, 2 paired-CTA tensor-core
+    int32_t kernel;            // 0 plain-FMA, 1 single-CTA tensor-core, 2 paired-CTA tensor-core, 3 the same over the 8-bit cache
     int32_t splits;
     int32_t cluster_merge, longest_first, fused_merge;
     int32_t device;
     size_t need, part_out, part_lse, counters;
     omni_mla_desc_t desc;
     const void *q, *kv;
-    alignas(64) CUtensorMap maps[4];
+    const float *kv_scale;     // 8-bit cache only
+    alignas(64) CUtensorMap maps[5];
 };
 static_assert(sizeof(LaunchPlan) <= sizeof(omni_mla_plan_t), "plan does not fit its public container");
 static_assert(alignof(LaunchPlan) <= 64, "plan alignment");
 
 static omni_status_t build_plan(const omni_mla_desc_t *desc, const void *q, const void *kv_cache, bool cached_maps,
-                                LaunchPlan *plan)
+                                LaunchPlan *plan, const float *kv_scale = nullptr, bool q8 = false)
 {
-    if (!desc || !q || !kv_cache) return OMNI_ERR_NULL;
+    if (!desc || !q || !kv_cache || (q8 && !kv_scale)) return OMNI_ERR_NULL;
     if (!desc_ok(desc)) return OMNI_ERR_SHAPE;
-    if (!aligned(q, 16) || !aligned(kv_cache, 128)) return OMNI_ERR_ALIGN;
+    // the 8-bit path exists for the paired-CTA kernel only (more than 64 heads, tensor cores)
+    if (q8 && !use_pair_kernel(desc)) return OMNI_ERR_SHAPE;
+    if (!aligned(q, 16) || !aligned(kv_cache, 128) || !aligned(kv_scale, 4)) return OMNI_ERR_ALIGN;
     const DeviceInfo &dev = device_info();
     if (!dev.ok) return OMNI_ERR_CUDA;
     if (dev.cc_major != 10) return OMNI_ERR_ARCH;
     plan->desc = *desc;
     plan->q = q;
     plan->kv = kv_cache;
+    plan->kv_scale = kv_scale;
     plan->device = dev.index;
-    plan->kernel = (desc->flags & OMNI_FLAG_SIMT) ? 0 : use_pair_kernel(desc) ? 2 : 1;
+    plan->kernel = q8 ? 3 : (desc->flags & OMNI_FLAG_SIMT) ? 0 : use_pair_kernel(desc) ? 2 : 1;
     const int splits = choose_splits(desc, dev.sm_count);
     plan->splits = splits;
     plan->part_out = part_out_bytes(desc, splits);
@@ -326,7 +331,7 @@ static omni_status_t build_plan(const omni_mla_desc_t *desc, const void *q, cons
     plan->cluster_merge = merge_in_cluster(desc, splits) ? 1 : 0;
     plan->fused_merge = (splits > 1 && merge_in_kernel(desc)) ? 1 : 0;
     // several waves of work units: start the longest requests first (the kernel ranks them itself)
-    plan->longest_first = (plan->kernel == 2 && !plan->cluster_merge && desc->batch <= 256 &&
+    plan->longest_first = (plan->kernel >= 2 && !plan->cluster_merge && desc->batch <= 256 &&
                            (long)desc->batch * splits > dev.sm_count / 2)
                               ? 1
                               : 0;
@@ -336,7 +341,9 @@ static omni_status_t build_plan(const omni_mla_desc_t *desc, const void *q, cons
     shape.num_pages = desc->num_pages;
     shape.batch = desc->batch;
     shape.heads = desc->num_heads;
-    if (plan->kernel == 2) {
+    if (plan->kernel == 3) {
+        if (!tc2q8_prepare_device() || !tc2q8_make_maps(shape, plan->maps, cached_maps)) return OMNI_ERR_CUDA;
+    } else if (plan->kernel == 2) {
         if (!tc2_prepare_device() || !tc2_make_maps(shape, plan->maps, cached_maps)) return OMNI_ERR_CUDA;
     } else if (plan->kernel == 1) {
         if (!tc_prepare_device() || !tc_make_maps(shape, plan->maps, cached_maps)) return OMNI_ERR_CUDA;
@@ -396,6 +403,7 @@ static omni_status_t run_plan(const LaunchPlan &plan, const int32_t *page_table,
     DecodeParams p;
     p.q = static_cast<const __nv_bfloat16 *>(plan.q);
     p.kv = static_cast<const __nv_bfloat16 *>(plan.kv);
+    p.kv_scale = plan.kv_scale;
     p.page_table = page_table;
     p.sel_idx = sel_idx;
     p.sel_len = sel_len;
@@ -432,7 +440,9 @@ static omni_status_t run_plan(const LaunchPlan &plan, const int32_t *page_table,
         simt_decode_kernel<<<grid, kSimtWarps * 32, 0, stream>>>(p);
         if (cudaPeekAtLastError() != cudaSuccess) st = OMNI_ERR_CUDA;
     } else {
-        st = plan.kernel == 2 ? tc2_launch(plan.maps, p, stream) : tc_launch(plan.maps, p, stream);
+        st = plan.kernel == 3   ? tc2q8_launch(plan.maps, p, stream)
+             : plan.kernel == 2 ? tc2_launch(plan.maps, p, stream)
+                                : tc_launch(plan.maps, p, stream);
     }
     if (st != OMNI_OK) return st;
     if (profile) cudaEventRecord(g_profile_after, stream);
@@ -460,6 +470,34 @@ static omni_status_t decode_impl(const omni_mla_desc_t *desc, const void *q, con
     if (st != OMNI_OK) return st;
     return run_plan(plan, page_table, sel_idx, sel_len, ctx_len, n_sink, n_recent, rolling, out, lse, workspace,
                     workspace_bytes, device_status, stream);
+}
+
+omni_status_t omni_sparse_mla_decode_q8(const omni_mla_desc_t *desc, const void *q, const void *kv_q8,
+                                        const float *kv_scale, const int32_t *page_table, const int32_t *sel_idx,
+                                        const int32_t *sel_len, void *out, float *lse, void *workspace,
+                                        size_t workspace_bytes, int32_t *device_status, void *stream)
+{
+    if (!desc || !q || !kv_q8 || !kv_scale || !page_table || !sel_idx || !sel_len || !out || !lse) return OMNI_ERR_NULL;
+    if (!desc_ok(desc) || !use_pair_kernel(desc)) return OMNI_ERR_SHAPE;
+    omni_status_t st = check_step_args(desc, page_table, sel_idx, sel_len, nullptr, 0, 0, false, out, lse);
+    if (st == OMNI_OK && (!aligned(q, 16) || !aligned(kv_q8, 128) || !aligned(kv_scale, 4))) st = OMNI_ERR_ALIGN;
+    if (st != OMNI_OK) return st;
+    LaunchPlan plan;
+    st = build_plan(desc, q, kv_q8, true, &plan, kv_scale, true);
+    if (st != OMNI_OK) return st;
+    return run_plan(plan, page_table, sel_idx, sel_len, nullptr, 0, 0, false, out, lse, workspace, workspace_bytes,
+                    device_status, stream);
+}
+
+omni_status_t omni_kv_quantize_q8(const void *kv_rows, int64_t num_rows, void *kv_q8, float *kv_scale, void *stream)
+{
+    if (!kv_rows || !kv_q8 || !kv_scale) return OMNI_ERR_NULL;
+    if (num_rows < 1 || num_rows > (int64_t)0x7fffffff * 8) return OMNI_ERR_SHAPE;
+    if (!aligned(kv_rows, 16) || !aligned(kv_q8, 128) || !aligned(kv_scale, 4)) return OMNI_ERR_ALIGN;
+    const unsigned blocks = (unsigned)((num_rows + 7) / 8);
+    quantize_q8_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const __nv_bfloat16 *>(kv_rows), num_rows, static_cast<uint8_t *>(kv_q8), kv_scale);
+    return cudaPeekAtLastError() == cudaSuccess ? OMNI_OK : OMNI_ERR_CUDA;
 }
 
 omni_status_t omni_sparse_mla_plan_init(const omni_mla_desc_t *desc, const void *q, const void *kv_cache,

@@ -19,7 +19,8 @@ constexpr float kLn2 = 0.6931471805599453f;
 // Everything a kernel needs to find its data; passed by value.
 struct DecodeParams {
     const __nv_bfloat16 *q;        // [B, H, 576]
-    const __nv_bfloat16 *kv;       // [num_pages * 64, 576]
+    const __nv_bfloat16 *kv;       // [num_pages * 64, 576]; the 8-bit kernel: bytes [num_pages * 64, 640]
+    const float *kv_scale;         // 8-bit cache only: one scale per pool row
     const int32_t *page_table;     // [B, max_pages]
     const int32_t *sel_idx;        // [B, max_sel]; null: the selection is Eq. 2's two ranges
     const int32_t *sel_len;        // [B]

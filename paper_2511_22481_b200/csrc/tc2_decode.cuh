@@ -263,7 +263,8 @@ __device__ __forceinline__ void tc_commit_pair_elect(uint64_t *bar, uint16_t bot
 // before the partner has said that its main loop is over (`ready_bar`, a remote arrive that the
 // partner fires as soon as its last P V has retired, while this CTA is still staging).
 // Called by every thread of the CTA after the main loop.
-__device__ __forceinline__ void cluster_merge_exchange(const DecodeParams &p, C2Control *ctl, uint8_t *smem,
+template <class Control>
+__device__ __forceinline__ void cluster_merge_exchange(const DecodeParams &p, Control *ctl, uint8_t *smem,
                                                        uint32_t tmem, int b, int s, uint32_t crank, int h0,
                                                        int head_rows, bool active, bool main_ok, float cm_lse, float cm_inv)
 {
@@ -379,6 +380,135 @@ __device__ __forceinline__ void cluster_merge_exchange(const DecodeParams &p, C2
     }
 }
 
+// An empty split (no tokens): zeros and -inf in place of a result.  Called by all threads.
+__device__ __forceinline__ void c2_store_empty(const DecodeParams &p, int b, int s, int h0, int head_rows, int warp, int lane)
+{
+    for (int r = warp; r < head_rows; r += kC2Threads / 32) {
+        const int h = h0 + r;
+        if (p.splits == 1) {
+            uint4 *o = reinterpret_cast<uint4 *>(p.out + ((size_t)b * p.heads + h) * kDv);
+            for (int i = lane; i < kDv * 2 / 16; i += 32) o[i] = make_uint4(0, 0, 0, 0);
+            if (lane == 0) p.lse[(size_t)b * p.heads + h] = -INFINITY;
+        } else {
+            const size_t u = ((size_t)b * p.splits + s) * p.heads + h;
+            float4 *o = reinterpret_cast<float4 *>(p.part_out + u * kDv);
+            for (int i = lane; i < kDv / 4; i += 32) o[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (lane == 0) p.part_lse[u] = -INFINITY;
+        }
+    }
+    if (p.splits > 1 && p.counters != nullptr) __threadfence();
+}
+
+// With more work units than the device runs at once, CTAs start in index order, so the requests
+// are taken longest first (ties by index): a long request that started last would otherwise run
+// on alone at the end.  Every CTA ranks the (at most 256) selection sizes itself: request j has
+// rank #{i : n_i > n_j, or n_i = n_j and i < j}, and the pair whose place in the grid is `slot`
+// takes the request of that rank.  lens: shared memory nobody uses yet (batch ints); flag: a
+// shared word.  Called by all threads; returns the request.
+__device__ __forceinline__ int c2_request_by_length_rank(const DecodeParams &p, int *lens, uint32_t *flag, int slot)
+{
+    for (int j = threadIdx.x; j < p.batch; j += kC2Threads) lens[j] = load_selection(p, j).n;
+    __syncthreads();
+    for (int j = threadIdx.x; j < p.batch; j += kC2Threads) {
+        const int nj = lens[j];
+        int before = 0;
+        for (int i = 0; i < p.batch; ++i) before += (lens[i] > nj) || (lens[i] == nj && i < j);
+        if (before == slot) *flag = (uint32_t)j;
+    }
+    __syncthreads();
+    const int b = (int)*flag;
+    __syncthreads();                                          // the shared memory is handed to the producers next
+    return b;
+}
+
+// Epilogue of a work unit whose result leaves through global memory (final bf16 rows, or fp32
+// partial rows of a split).  Each of the eight softmax warps owns 32 rows x 128 value columns
+// of the accumulator: warp quarter q = warp % 4 serves head rows 32 * (q % 2) + lane and value
+// columns 256 * (q / 2) + 128 * sub + [0, 128), sub = 1 for warps 8-11.  It moves them out in
+// rounds of 128 bytes per row: tensor memory -> registers (scaled by 1 / lt) -> a warp-private
+// staging tile in shared memory (all operand buffers are dead by now; 144-byte pitch, so
+// neither the row-per-lane writes nor the line-per-8-lanes reads conflict) -> global memory as
+// whole 128-byte lines, four rows per instruction.  The staging tile is double buffered and no
+// CTA-wide barrier is needed, so the stores of one round overlap the tensor-memory reads of the
+// next.  lt: the row's sum of weights; m_ref: its reference maximum (log2 units).
+__device__ __forceinline__ void c2_store_result(const DecodeParams &p, uint8_t *smem, uint32_t tmem, int warp, int lane,
+                                                int b, int s, int h0, int head_rows, float lt, float m_ref)
+{
+    const int quarter = warp & 3;
+    const int sub = warp >= 8 ? 1 : 0;
+    const int row = (quarter & 1) * 32 + lane;
+    const int part = (quarter >> 1) * 2 + sub;
+    const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+    const float inv = lt > 0.f ? 1.f / lt : 0.f;
+    const int h = h0 + row;
+    const bool final_out = p.splits == 1;
+    const size_t u = final_out ? ((size_t)b * p.heads + h) : (((size_t)b * p.splits + s) * p.heads + h);
+    constexpr uint32_t kStagePitch = 144, kStageBytes = 32 * kStagePitch;
+    const int widx = sub * 4 + ((warp - 2) & 3);                         // 0..7
+    uint8_t *stage = smem + (size_t)widx * 2 * kStageBytes;
+    const uint32_t row_bytes = final_out ? kDv * 2 : kDv * 4;
+    const int row0 = (quarter & 1) * 32;                                  // first head row of this warp
+    // global address of (row0, this warp's first value column)
+    const size_t u0 = final_out ? ((size_t)b * p.heads + h0 + row0) : (((size_t)b * p.splits + s) * p.heads + h0 + row0);
+    uint8_t *gbase = (final_out ? reinterpret_cast<uint8_t *>(p.out + u0 * kDv)
+                                : reinterpret_cast<uint8_t *>(p.part_out + u0 * kDv)) + part * (row_bytes / 4);
+    const int rows_here = max(0, min(32, head_rows - row0));              // rows of this warp that exist
+    const int rounds = final_out ? 2 : 4;
+#pragma unroll 1
+    for (int q = 0; q < rounds; ++q) {
+        uint8_t *buf = stage + (q & 1) * kStageBytes;
+        uint4 *mine = reinterpret_cast<uint4 *>(buf + lane * kStagePitch);
+        __syncwarp();
+        if (final_out) {
+            // 64 columns -> 128 bytes of bf16
+#pragma unroll
+            for (int c2 = 0; c2 < 2; ++c2) {
+                uint32_t ov[32];
+                tc_ld32(tmem + lane_base + kColO + 128 * sub + q * 64 + c2 * 32, ov);
+                tc_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    uint4 w;
+                    w.x = pack_bf16(__uint_as_float(ov[8 * j]) * inv, __uint_as_float(ov[8 * j + 1]) * inv);
+                    w.y = pack_bf16(__uint_as_float(ov[8 * j + 2]) * inv, __uint_as_float(ov[8 * j + 3]) * inv);
+                    w.z = pack_bf16(__uint_as_float(ov[8 * j + 4]) * inv, __uint_as_float(ov[8 * j + 5]) * inv);
+                    w.w = pack_bf16(__uint_as_float(ov[8 * j + 6]) * inv, __uint_as_float(ov[8 * j + 7]) * inv);
+                    mine[c2 * 4 + j] = w;
+                }
+            }
+        } else {
+            // 32 columns -> 128 bytes of fp32
+            uint32_t ov[32];
+            tc_ld32(tmem + lane_base + kColO + 128 * sub + q * 32, ov);
+            tc_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                mine[j] = make_uint4(__float_as_uint(__uint_as_float(ov[4 * j]) * inv),
+                                     __float_as_uint(__uint_as_float(ov[4 * j + 1]) * inv),
+                                     __float_as_uint(__uint_as_float(ov[4 * j + 2]) * inv),
+                                     __float_as_uint(__uint_as_float(ov[4 * j + 3]) * inv));
+        }
+        __syncwarp();
+        uint8_t *gq = gbase + q * 128;
+        uint4 v[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+            v[k] = *reinterpret_cast<const uint4 *>(buf + (4 * k + (lane >> 3)) * kStagePitch + (lane & 7) * 16);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const int r = 4 * k + (lane >> 3);
+            if (r < rows_here) *reinterpret_cast<uint4 *>(gq + (size_t)r * row_bytes + (lane & 7) * 16) = v[k];
+        }
+    }
+    if (h < p.heads && part == 0) {
+        const float lse = lt > 0.f ? (m_ref + log2f(lt)) * kLn2 : -INFINITY;
+        if (final_out)
+            p.lse[u] = lse;
+        else
+            p.part_lse[u] = lse;
+    }
+}
+
 __global__ void __launch_bounds__(kC2Threads, 1)
 tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
                   const __grid_constant__ CUtensorMap kv_k_map, const __grid_constant__ CUtensorMap kv_v_map,
@@ -447,25 +577,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
     // may be scheduled as soon as resources allow; it waits in the same way before it reads.
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (p.longest_first) {
-        // The grid runs in several waves and CTAs start in index order, so the requests are
-        // taken longest first (ties by index): a long request that started last would otherwise
-        // run on alone at the end.  Every CTA ranks the (at most 256) selection sizes itself:
-        // request j has rank #{i : n_i > n_j, or n_i = n_j and i < j}, and this pair takes the
-        // request whose rank is its own place in the grid.
-        int *lens = reinterpret_cast<int *>(smem);               // operand tiles are not in use yet
-        for (int j = threadIdx.x; j < p.batch; j += kC2Threads) lens[j] = load_selection(p, j).n;
-        __syncthreads();
-        for (int j = threadIdx.x; j < p.batch; j += kC2Threads) {
-            const int nj = lens[j];
-            int before = 0;
-            for (int i = 0; i < p.batch; ++i) before += (lens[i] > nj) || (lens[i] == nj && i < j);
-            if (before == b) ctl->merge_flag = (uint32_t)j;
-        }
-        __syncthreads();
-        b = (int)ctl->merge_flag;
-        __syncthreads();                                          // smem is handed to the producers next
-    }
+    if (p.longest_first) b = c2_request_by_length_rank(p, reinterpret_cast<int *>(smem), &ctl->merge_flag, b);
     const Selection selection = load_selection(p, b);
     const int n = selection.n;
     const bool bad_len = selection.bad;
@@ -477,20 +589,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
     if (!active && bad_len && threadIdx.x == 0 && crank == 0) flag_status(p.status, OMNI_DEV_BAD_INDEX);
     if (!active && !p.cluster_merge) {
         // empty split (the same decision in both CTAs of the pair): zeros and -inf, no pipeline
-        for (int r = warp; r < head_rows; r += kC2Threads / 32) {
-            const int h = h0 + r;
-            if (p.splits == 1) {
-                uint4 *o = reinterpret_cast<uint4 *>(p.out + ((size_t)b * p.heads + h) * kDv);
-                for (int i = lane; i < kDv * 2 / 16; i += 32) o[i] = make_uint4(0, 0, 0, 0);
-                if (lane == 0) p.lse[(size_t)b * p.heads + h] = -INFINITY;
-            } else {
-                const size_t u = ((size_t)b * p.splits + s) * p.heads + h;
-                float4 *o = reinterpret_cast<float4 *>(p.part_out + u * kDv);
-                for (int i = lane; i < kDv / 4; i += 32) o[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (lane == 0) p.part_lse[u] = -INFINITY;
-            }
-        }
-        if (p.splits > 1 && p.counters != nullptr) __threadfence();
+        c2_store_empty(p, b, s, h0, head_rows, warp, lane);
     }
 
     const uint32_t tmem = ctl->tmem_base;
@@ -963,84 +1062,11 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
             cm_inv = lt > 0.f ? 1.f / lt : 0.f;
             cm_lse = lt > 0.f ? (m_ref + log2f(lt)) * kLn2 : -INFINITY;
         } else if (ok) {
-            // Each warp owns 32 rows x 128 value columns of the result.  It moves them out in rounds
-            // of 128 bytes per row: tensor memory -> registers (scaled) -> a warp-private staging
-            // tile in shared memory (all operand buffers are dead by now; 144-byte pitch, so neither
-            // the row-per-lane writes nor the line-per-8-lanes reads conflict) -> global memory as
-            // whole 128-byte lines, four rows per instruction.  The staging tile is double
-            // buffered and no CTA-wide barrier is needed, so the stores of one round overlap the
-            // tensor-memory reads of the next.
             tc_fence_after();
             const float lt = (ctl->xchg[tiles & 1][0][row] + ctl->xchg[tiles & 1][1][row]) +
                              (ctl->xchg[tiles & 1][2][row] + ctl->xchg[tiles & 1][3][row]);
-            const float inv = lt > 0.f ? 1.f / lt : 0.f;
-            const int h = h0 + row;
+            c2_store_result(p, smem, tmem, warp, lane, b, s, h0, head_rows, lt, m_ref);
             const bool final_out = p.splits == 1;
-            const size_t u = final_out ? ((size_t)b * p.heads + h) : (((size_t)b * p.splits + s) * p.heads + h);
-            constexpr uint32_t kStagePitch = 144, kStageBytes = 32 * kStagePitch;
-            const int widx = sub * 4 + ((warp - 2) & 3);                         // 0..7
-            uint8_t *stage = smem + (size_t)widx * 2 * kStageBytes;
-            const uint32_t row_bytes = final_out ? kDv * 2 : kDv * 4;
-            const int row0 = (quarter & 1) * 32;                                  // first head row of this warp
-            // global address of (row0, this warp's first value column)
-            const size_t u0 = final_out ? ((size_t)b * p.heads + h0 + row0) : (((size_t)b * p.splits + s) * p.heads + h0 + row0);
-            uint8_t *gbase = (final_out ? reinterpret_cast<uint8_t *>(p.out + u0 * kDv)
-                                        : reinterpret_cast<uint8_t *>(p.part_out + u0 * kDv)) + part * (row_bytes / 4);
-            const int rows_here = max(0, min(32, head_rows - row0));              // rows of this warp that exist
-            const int rounds = final_out ? 2 : 4;
-#pragma unroll 1
-            for (int q = 0; q < rounds; ++q) {
-                uint8_t *buf = stage + (q & 1) * kStageBytes;
-                uint4 *mine = reinterpret_cast<uint4 *>(buf + lane * kStagePitch);
-                __syncwarp();
-                if (final_out) {
-                    // 64 columns -> 128 bytes of bf16
-#pragma unroll
-                    for (int c2 = 0; c2 < 2; ++c2) {
-                        uint32_t ov[32];
-                        tc_ld32(tmem + lane_base + kColO + 128 * sub + q * 64 + c2 * 32, ov);
-                        tc_wait_ld();
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            uint4 w;
-                            w.x = pack_bf16(__uint_as_float(ov[8 * j]) * inv, __uint_as_float(ov[8 * j + 1]) * inv);
-                            w.y = pack_bf16(__uint_as_float(ov[8 * j + 2]) * inv, __uint_as_float(ov[8 * j + 3]) * inv);
-                            w.z = pack_bf16(__uint_as_float(ov[8 * j + 4]) * inv, __uint_as_float(ov[8 * j + 5]) * inv);
-                            w.w = pack_bf16(__uint_as_float(ov[8 * j + 6]) * inv, __uint_as_float(ov[8 * j + 7]) * inv);
-                            mine[c2 * 4 + j] = w;
-                        }
-                    }
-                } else {
-                    // 32 columns -> 128 bytes of fp32
-                    uint32_t ov[32];
-                    tc_ld32(tmem + lane_base + kColO + 128 * sub + q * 32, ov);
-                    tc_wait_ld();
-#pragma unroll
-                    for (int j = 0; j < 8; ++j)
-                        mine[j] = make_uint4(__float_as_uint(__uint_as_float(ov[4 * j]) * inv),
-                                             __float_as_uint(__uint_as_float(ov[4 * j + 1]) * inv),
-                                             __float_as_uint(__uint_as_float(ov[4 * j + 2]) * inv),
-                                             __float_as_uint(__uint_as_float(ov[4 * j + 3]) * inv));
-                }
-                __syncwarp();
-                uint8_t *gq = gbase + q * 128;
-                uint4 v[8];
-#pragma unroll
-                for (int k = 0; k < 8; ++k)
-                    v[k] = *reinterpret_cast<const uint4 *>(buf + (4 * k + (lane >> 3)) * kStagePitch + (lane & 7) * 16);
-#pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    const int r = 4 * k + (lane >> 3);
-                    if (r < rows_here) *reinterpret_cast<uint4 *>(gq + (size_t)r * row_bytes + (lane & 7) * 16) = v[k];
-                }
-            }
-            if (h < p.heads && part == 0) {
-                const float lse = lt > 0.f ? (m_ref + log2f(lt)) * kLn2 : -INFINITY;
-                if (final_out)
-                    p.lse[u] = lse;
-                else
-                    p.part_lse[u] = lse;
-            }
             // with the in-kernel merge the partial results must be visible before this CTA is counted
             if (!final_out && p.counters != nullptr) __threadfence();
         }

@@ -83,3 +83,54 @@ def check_workload(w, flags=0, num_splits=0, reqs=None, heads=None, what="", str
     g = plan.out.cpu()[r][:, h]
     gl = plan.lse.cpu()[r][:, h]
     return compare(g, gl, ref_out, ref_lse, what, strict_abs), plan
+
+
+# ------------------------------------------------------------------ 8-bit latent cache
+
+def quantise_pool_q8(w, check_rows=4096, seed=0):
+    """8-bit form of a workload's pool.  The pool is quantised on the device through the C ABI
+    and the result is compared, bit for bit, with the oracle's quantiser on `check_rows` rows
+    (all rows of a small pool), so the decode tests run on a cache the oracle vouches for."""
+    from oracle import q8
+    rows = w.kv_cache.view(-1, w.d_qk)
+    n = rows.shape[0]
+    cache = torch.empty((n, B.OMNI_Q8_ROW_BYTES), dtype=torch.uint8, device=rows.device)
+    scale = torch.empty((n,), dtype=torch.float32, device=rows.device)
+    B.omni_kv_quantize_q8(rows, cache, scale)
+    torch.cuda.synchronize()
+    pick = np.arange(n) if n <= check_rows else np.sort(np.random.default_rng(seed).choice(n, check_rows, replace=False))
+    idx = torch.from_numpy(pick).to(rows.device)
+    bits = rows[idx].cpu().view(torch.int16).numpy().view(np.uint16)
+    want_cache, want_scale = q8.quantise_rows(bits)
+    assert np.array_equal(scale[idx].cpu().numpy().view(np.uint32), want_scale.view(np.uint32)), "scales differ"
+    assert np.array_equal(cache[idx].cpu().numpy(), want_cache), "codes differ"
+    return cache, scale
+
+
+def oracle_subset_q8(w, cache, scale, reqs=None, heads=None):
+    """Oracle results over the de-quantised rows, for the listed requests and heads."""
+    from oracle import q8
+    reqs = list(range(w.batch)) if reqs is None else list(reqs)
+    heads = list(range(w.heads)) if heads is None else list(heads)
+    pt = w.page_table.cpu().numpy()[reqs]
+    si = w.sel_idx.cpu().numpy()[reqs]
+    sl = w.sel_len.cpu().numpy()[reqs]
+    rows = oracle.resolve_rows(pt, si, sl, w.page_size, w.num_pages)
+    gather = torch.from_numpy(np.where(rows < 0, 0, rows)).to(cache.device).view(-1)
+    krows = q8.dequantise_rows(cache[gather].cpu().numpy(), scale[gather].cpu().numpy()).reshape(len(reqs), -1, w.d_qk)
+    q = w.q[torch.tensor(reqs, device=w.q.device)][:, torch.tensor(heads, device=w.q.device)].cpu().to(torch.float64).numpy()
+    return q8.attend_dequantised(q, krows, sl, w.d_v, w.scale)
+
+
+def check_workload_q8(w, flags=0, num_splits=0, reqs=None, heads=None, what="", strict_abs=False, quantised=None):
+    cache, scale = quantised or quantise_pool_q8(w)
+    plan = B.plan_for(w, num_splits=num_splits, flags=flags)
+    plan.status.zero_()
+    B.omni_sparse_mla_decode_q8(plan.desc, w.q, cache, scale, w.page_table, w.sel_idx, w.sel_len, plan.out, plan.lse,
+                                plan.workspace, plan.status)
+    torch.cuda.synchronize()
+    assert int(plan.status.item()) == 0, what + ": device status %d" % int(plan.status.item())
+    ref_out, ref_lse = oracle_subset_q8(w, cache, scale, reqs, heads)
+    r = torch.arange(w.batch) if reqs is None else torch.tensor(list(reqs))
+    h = torch.arange(w.heads) if heads is None else torch.tensor(list(heads))
+    return compare(plan.out.cpu()[r][:, h], plan.lse.cpu()[r][:, h], ref_out, ref_lse, what, strict_abs), plan

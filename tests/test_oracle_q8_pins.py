@@ -59,10 +59,10 @@ def test_quantiser_on_hand_worked_rows():
     row[1, 7] = -3.5                               # amax 3.5 -> scale 3.5/448 = 2^-7: -3.5/scale = -448
     row[1, 8] = 1.75                               # 224
     row[1, 9] = 2.0 ** -7                          # 1.0 after scaling
-    # row 2 stays all zero: scale is defined as 1, every code 0
+    # row 2 stays all zero: amax is floored at 2^-60, every code 0
     cache, scale = q8.quantise_rows(_bits(row))
     assert cache.shape == (3, 640) and scale.dtype == np.float32
-    assert scale.tolist() == [1.0, 3.5 / 448.0, 1.0]
+    assert scale.tolist() == [1.0, 3.5 / 448.0, float(np.float32(2.0 ** -60) / np.float32(448.0))]
     assert cache[0, :4].tolist() == [0x7E, 0xF6, 0x38, 0x2E]
     assert cache[1, 7] == 0xFE and cache[1, 8] == 0x76 and cache[1, 9] == 0x38
     assert not cache[2, :512].any() and not cache[1, :7].any()
