@@ -163,7 +163,7 @@ def _oracle_sample(w, target_s=15.0, max_requests=None):
                 f32_seconds=f32_seconds, f32_tokens=int(sl.sum()))
 
 
-WORKLOAD_HELP = ("config2 (default, the named benchmark) | config1 | config3 | config4 | "
+WORKLOAD_HELP = ("config2 (default, the named benchmark) | config1 | config3[:<batch>] | config4 | "
                  "config5:<batch>:<selected>[:dense] (one sweep cell) | "
                  "eq2:<batch>:<n_sink>:<n_recent>[:list] (the paper's sink + recent rule on 32768-token contexts, "
                  "through the range entry point, or with :list through the index-list entry point) | "
@@ -172,9 +172,14 @@ WORKLOAD_HELP = ("config2 (default, the named benchmark) | config1 | config3 | c
 
 
 def make_workload(spec, dev, batch):
-    """Build a named workload and a one-line description of it."""
+    """Build a named workload and a one-line description of it.  A trailing ":q8" runs the same
+    selection over the 8-bit form of the same pool (omni_sparse_mla_decode_q8)."""
     import numpy as np
     from paper_2511_22481_b200 import workloads as W
+    if spec.endswith(":q8"):
+        w, text = make_workload(spec[:-3], dev, batch)
+        w.meta["entry"] = "q8"
+        return w, text + "; 8-bit latent cache (640-byte rows: 512 E4M3 codes + 64 bf16 rope columns, one fp32 scale per row)"
     if spec == "config2":
         w = W.config2_r1(dev, batch=batch)
         text = ("config2 DeepSeek-R1-shaped decode: batch %d/GPU, 128 heads, d_qk 576, d_v 512, ctx 32768, "
@@ -182,9 +187,10 @@ def make_workload(spec, dev, batch):
     elif spec == "config1":
         w = W.config1_tiny(dev)
         text = "config1 tiny: batch 1, 16 heads, ctx 4096, identity page table, 832 selected tokens, seed 0"
-    elif spec == "config3":
-        w = W.config3_ragged(dev)
-        text = "config3 ragged: batch 128, 128 heads, ctx U[4096,65536], 1/8 of pages selected, seed 2"
+    elif spec == "config3" or spec.startswith("config3:"):
+        n3 = int(spec.split(":")[1]) if ":" in spec else 128          # config3:<batch>: the first requests only (profiling)
+        w = W.config3_ragged(dev, batch=n3)
+        text = "config3 ragged: batch %d, 128 heads, ctx U[4096,65536], 1/8 of pages selected, seed 2" % n3
     elif spec == "config4":
         w = W.config4_topk(dev)
         text = "config4 token-level top-k: batch 16, 128 heads, ctx 131072, 2048 scattered tokens/request, seed 3"
@@ -365,9 +371,22 @@ def main():
     clones = max(2, args.clones)
     while clones > 2 and clones * w.kv_cache.numel() * 2 > 40e9:      # keep the rotated copies within 40 GB
         clones -= 1
-    pools = [w.kv_cache] + [w.kv_cache.clone() for _ in range(clones - 1)]
+    q8 = w.meta.get("entry") == "q8"
+    if q8:
+        # the same pool in its 8-bit form; the bf16 copy is released
+        rows = w.kv_cache.view(-1, w.d_qk)
+        cache = torch.empty((rows.shape[0], B.OMNI_Q8_ROW_BYTES), dtype=torch.uint8, device=dev)
+        scale = torch.empty((rows.shape[0],), dtype=torch.float32, device=dev)
+        B.omni_kv_quantize_q8(rows, cache, scale)
+        torch.cuda.synchronize()
+        w.kv_cache = None
+        pools = [(cache, scale)] + [(cache.clone(), scale.clone()) for _ in range(clones - 1)]
+    else:
+        pools = [w.kv_cache] + [w.kv_cache.clone() for _ in range(clones - 1)]
     plan = B.plan_for(w, flags=flags)
-    kv_bytes = w.selected_kv_bytes
+    # algorithmic bytes per selected token: the row as stored (and, for the 8-bit cache, its scale)
+    row_bytes = (B.OMNI_Q8_ROW_BYTES + 4) if q8 else KV_ROW_BYTES
+    kv_bytes = w.selected_tokens * row_bytes
     flops = w.selected_tokens * w.heads * FLOP_PER_TOKEN_HEAD
     launches_per_step = B.omni_sparse_mla_num_launches(plan.desc)
 
@@ -380,7 +399,13 @@ def main():
     # once (split plan, tensor maps), and the per-step C call with its arguments marshalled once,
     # so that a step costs the host one foreign call and one kernel launch.
     planned = None
-    if not ranges:
+    if q8:
+        def q8_call(pool):
+            cache_i, scale_i = pool
+            return lambda: B.omni_sparse_mla_decode_q8(plan.desc, w.q, cache_i, scale_i, w.page_table, w.sel_idx, w.sel_len,
+                                                       plan.out, plan.lse, plan.workspace, plan.status)
+        planned = [q8_call(pool) for pool in pools]
+    elif not ranges:
         stream = torch.cuda.current_stream()
         planned = [B.bind_planned(B.omni_sparse_mla_plan_init(plan.desc, w.q, pool), w.page_table, w.sel_idx,
                                   w.sel_len, plan.out, plan.lse, plan.workspace, plan.status, stream)
@@ -447,9 +472,22 @@ def main():
     h2d = sum(t.numel() * t.element_size() for t in (q_h, pt_h, si_h, sl_h))
     d2h = sum(t.numel() * t.element_size() for t in (out_h, lse_h))
 
-    def e2e_step(i):
-        B.omni_sparse_mla_decode_host(plan.desc, q_h, pools[i % clones], pt_h, si_h, sl_h, out_h,
-                                      lse_h, staging, plan.workspace, plan.status)
+    if q8:
+        # no host-buffer entry point for the 8-bit cache: the same copies issued around the device call
+        q_d, pt_d, si_d, sl_d = (torch.empty_like(t, device=dev) for t in (q_h, pt_h, si_h, sl_h))
+
+        def e2e_step(i):
+            for dst, src in ((q_d, q_h), (pt_d, pt_h), (si_d, si_h), (sl_d, sl_h)):
+                dst.copy_(src, non_blocking=True)
+            cache_i, scale_i = pools[i % clones]
+            B.omni_sparse_mla_decode_q8(plan.desc, q_d, cache_i, scale_i, pt_d, si_d, sl_d, plan.out, plan.lse,
+                                        plan.workspace, plan.status)
+            out_h.copy_(plan.out, non_blocking=True)
+            lse_h.copy_(plan.lse, non_blocking=True)
+    else:
+        def e2e_step(i):
+            B.omni_sparse_mla_decode_host(plan.desc, q_h, pools[i % clones], pt_h, si_h, sl_h, out_h,
+                                          lse_h, staging, plan.workspace, plan.status)
 
     e2e_steps = args.steps
     for i in range(args.warmup):
@@ -488,11 +526,13 @@ def main():
             "value": round(value, 2), "unit": "GB/s", "us_per_step": round(ms_per_step * 1e3, 3),
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": round(ms_per_step, 6), "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "vs_baseline": None, "dtype": "e4m3 cache, bf16 q and out, fp32 accumulate" if q8 else "bf16", "data": "synthetic",
             "config": {"workload": workload_text,
                        "selected_tokens_per_gpu": w.selected_tokens, "kv_bytes_per_step_per_gpu": kv_bytes,
+                       "kv_bytes_per_token": row_bytes,
                        "splits": plan.splits, "kernel": args.kernel, "launches_per_step": launches_per_step,
-                       "entry": "omni_sparse_mla_decode_planned" if planned is not None else "range entry point",
+                       "entry": ("omni_sparse_mla_decode_q8" if q8 else "omni_sparse_mla_decode_planned" if planned is not None
+                                 else "range entry point"),
                        "l2": "cold: %d pool copies rotated (%.0f MB touched per cycle vs %.0f MB L2)"
                              % (clones, clones * kv_bytes / 1e6, L2_BYTES / 1e6),
                        "parallelism": "dp%d (independent requests, no collective)" % world},
@@ -523,7 +563,7 @@ def main():
                          "frac_of_nominal_8TBs": round(achieved / 8000.0, 4),
                          "kernel_source_hash": khash},
         }
-        if world == 1 and not args.no_cpu_baseline:
+        if world == 1 and not args.no_cpu_baseline and not q8:
             s = _oracle_sample(w)
             cpu_value = s["tokens"] * KV_ROW_BYTES / s["seconds"] / 1e9
             line["cpu_baseline"] = {

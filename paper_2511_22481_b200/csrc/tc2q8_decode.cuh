@@ -545,10 +545,8 @@ tc2q8_decode_kernel(const __grid_constant__ CUtensorMap q_nope_map, const __grid
             };
             bool ok = mbar_wait(&ctl->q_ready, 0);
             ok = __all_sync(0xffffffffu, ok);
-            if (ok) {
-                tc_fence_after();
-                ok = qk_tile(0);
-            }
+            if (ok) tc_fence_after();
+            if (ok) ok = qk_tile(0);
             if (ok && tiles_u > 1) ok = qk_tile(1);
             for (int i = 0; ok && i < tiles_u; ++i) {
                 if (i + 2 < tiles_u) ok = qk_tile(i + 2);
