@@ -402,7 +402,10 @@ omni_status_t omni_sparse_mla_decode_host(const omni_mla_desc_t *desc, const voi
  *     the batch, or use omni_sparse_mla_decode with a workspace of your own);
  *   - the first call on each device looks up the array's device address (one runtime query,
  *     with that device current) and caches it; make that first call during start-up, before
- *     any stream capture begins;
+ *     any stream capture begins AND before the process hands the rest of the device memory to
+ *     its own pools: the CUDA runtime may load the library's device image, array included,
+ *     only at that first query, and a device with no free memory left then fails it
+ *     (OMNI_ERR_CUDA);
  *   - all calls on one device share the one array, which keeps whatever the previous call left
  *     in it.  The caller clears nothing (each call overwrites every partial result it reads
  *     back and clears the few counters it needs at zero itself), but two calls that overlap on the GPU, e.g. on different streams, race on
