@@ -25,8 +25,9 @@
 // issues one every 25-64 clocks).  Completion is broadcast to both CTAs with multicast commits.
 //
 // Warps per CTA: 0 K-role producer, 1 MMA issuer (CTA 0 only) + tensor-memory owner,
-// 2-5 and 8-11 softmax / epilogue (two warps per tensor-memory lane quarter, 16 of a tile's 64
-// tokens per thread), 6 V-role producer, 7 L2 prefetcher (CTA 0 only): shared memory holds
+// 2-5 and 8-11 softmax / epilogue (two groups of four warps that take the tiles in turn: warps
+// 2-5 the even tiles, 8-11 the odd ones, 32 of a tile's 64 tokens per thread; all eight share
+// the epilogue), 6 V-role producer, 7 L2 prefetcher (CTA 0 only): shared memory holds
 // only two tiles, about one HBM latency of work, so each whole page is pulled into L2 one tile
 // before its K-role load and the shared-memory refills start from a line already on its way.
 //
@@ -37,9 +38,10 @@
 //   columns 256..287  S buffer 0: lane L, column x <-> head row L%64, token 32*(L/64) + x
 //   columns 288..319, 320..351  S buffers 1, 2 (Q K^T runs two tiles ahead of P V)
 //
-// With more than one split per request the last CTA to finish a request's head half merges the
-// partial results itself (a counter per (request, head half) in the workspace), so a decode
-// call is one launch.
+// Splits of a request are merged in one of three ways chosen by the host: inside a cluster of
+// two pairs (two splits, see cluster_merge_exchange), by a separate merge kernel over fp32
+// partial results, or by the last CTA to finish a request's head half (a counter per (request,
+// head half) in the workspace).
 #pragma once
 
 #include <type_traits>
@@ -81,10 +83,10 @@ struct C2Control {
     uint64_t s_empty[3];
     uint64_t p_full[2];
     uint64_t pv_done[2];                 // P V of a tile retired: frees its V stage and its P buffer
-    uint64_t x_bar;                      // softmax threads: row-maximum exchange
+    uint64_t x_bar;                      // all softmax threads: exchange of the final row sums
     uint64_t exit_bar;                   // both CTAs of the pair are done with tensor memory
     uint64_t valid_mask[kMaskRing];      // per tile: validity of its 64 tokens
-    float xchg[2][4][64];                // [tile parity][token quarter][head row]
+    float xchg[2][4][64];                // row maxima: [group][parity of the group's tile][token half][head row]; at the end [0][thread of the row][head row]: row sums
     uint32_t tmem_base;
     uint32_t abort;
     uint32_t merge_flag;
@@ -92,7 +94,9 @@ struct C2Control {
     int32_t k_progress;                  // tiles whose K loads the producer has started (L2 prefetch pacing)
     uint64_t recv_bar;                   // cluster merge: the partner's block has arrived
     uint64_t ready_bar;                  // cluster merge: the partner's main loop is over
-    float xlse[2][64];                   // cluster merge: log-sum-exp of either split, per head row
+    uint64_t xg_bar[2];                  // row-maximum exchange inside either softmax group
+    uint64_t ref_bar;                    // the reference maxima after a tile are published (4 warps of its group)
+    float ref[2][64];                    // [tile parity][head row]: running reference maximum after that tile
 };
 static_assert(sizeof(C2Control) <= kC2SmemCtlBytes, "control block too large");
 static_assert(kC2SmemBytes <= 232448, "shared memory budget");
@@ -272,8 +276,9 @@ __device__ __forceinline__ void cluster_merge_exchange(const DecodeParams &p, Co
     constexpr uint32_t kPitch = kSliceBytes + 16;        // row-per-lane 16-byte accesses do not conflict
     constexpr uint32_t kRowsBytes = 64 * kPitch;         // 66,560
     constexpr uint32_t kBlockBytes = kRowsBytes + 256;   // + 64 log-sum-exps
-    static_assert(3 * kBlockBytes <= kC2SmemCtl, "exchange tiles must fit below the control block");
+    static_assert(3 * kBlockBytes + 512 <= kC2SmemCtl, "exchange tiles must fit below the control block");
     uint8_t *send = smem, *keep = smem + kBlockBytes, *recv = smem + 2 * kBlockBytes;
+    float(*xlse)[64] = reinterpret_cast<float(*)[64]>(smem + 3 * kBlockBytes);   // weights of the two splits per head row
     const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;
     const bool is_softmax = (warp >= 2 && warp <= 5) || warp >= 8;
     if (!is_softmax) return;
@@ -354,8 +359,8 @@ __device__ __forceinline__ void cluster_merge_exchange(const DecodeParams &p, Co
             if (cm_lse > -INFINITY) w_own = exp2f((cm_lse - total) * kLog2e);
             if (other > -INFINITY) w_other = exp2f((other - total) * kLog2e);
         }
-        ctl->xlse[0][row] = w_own;
-        ctl->xlse[1][row] = w_other;
+        xlse[0][row] = w_own;
+        xlse[1][row] = w_other;
         if (s == 0 && row < head_rows) p.lse[(size_t)b * p.heads + h0 + row] = total;
     }
     asm volatile("bar.sync 1, 256;" ::: "memory");
@@ -363,7 +368,7 @@ __device__ __forceinline__ void cluster_merge_exchange(const DecodeParams &p, Co
     const int t = (sub * 4 + ((warp - 2) & 3)) * 32 + lane;          // 0..255
     for (int item = t; item < head_rows * 32; item += 256) {
         const int r = item >> 5, c = item & 31;
-        const float wk = ctl->xlse[0][r], wr = ctl->xlse[1][r];
+        const float wk = xlse[0][r], wr = xlse[1][r];
         const uint4 *k4 = reinterpret_cast<const uint4 *>(keep + (size_t)r * kPitch + c * 32);
         const uint4 *r4 = reinterpret_cast<const uint4 *>(recv + (size_t)r * kPitch + c * 32);
         const uint4 k0 = k4[0], k1 = k4[1], r0 = r4[0], r1 = r4[1];
@@ -541,17 +546,22 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
     // programmatic dependent launch it overlaps the tail of the kernel before this one) --------
     if (threadIdx.x == 0) {
         mbar_init(&ctl->q_full, 1);
+        // arrivals per tile on the pair's score / weight barriers: one per softmax warp that works on
+        // the tile, in either CTA (the four warps of the tile's group)
+        constexpr uint32_t kTileWarps = 8;
         for (int i = 0; i < 2; ++i) {
             mbar_init(&ctl->k_full[i], 1);
             mbar_init(&ctl->k_empty[i], 1);
             mbar_init(&ctl->v_full[i], 1);
-            mbar_init(&ctl->p_full[i], 16);
+            mbar_init(&ctl->p_full[i], kTileWarps);
             mbar_init(&ctl->pv_done[i], 1);
+            mbar_init(&ctl->xg_bar[i], 128);
         }
         for (int i = 0; i < 3; ++i) {
             mbar_init(&ctl->s_full[i], 1);
-            mbar_init(&ctl->s_empty[i], 16);     // one arrival per softmax warp of either CTA
+            mbar_init(&ctl->s_empty[i], kTileWarps);
         }
+        mbar_init(&ctl->ref_bar, 4);
         mbar_init(&ctl->x_bar, 256);
         mbar_init(&ctl->exit_bar, 2);
         mbar_init(&ctl->recv_bar, 1);
@@ -928,11 +938,10 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
         __syncwarp();
     } else {
         // =========================== softmax + epilogue =================================
-        // Eight warps (2-5 and 8-11): two per tensor-memory lane quarter.  A thread serves head row
-        // L % 64 (L = its tensor-memory lane), the token half L / 64 of the tile and, within that
-        // half, the 16 tokens picked by `sub` (0 for warps 2-5, 1 for warps 8-11); of O it serves
-        // value columns 256 * (L / 64) + 128 * sub + [0, 128).  The four threads of a row exchange
-        // their partial row maximum through shared memory.
+        // Eight warps (2-5 and 8-11): two per tensor-memory lane quarter, one in each of two groups
+        // (sub = 0 for warps 2-5, 1 for warps 8-11).  A thread serves head row L % 64 (L = its
+        // tensor-memory lane); in the epilogue it owns value columns 256 * (L / 64) + 128 * sub +
+        // [0, 128) of that row.
         const int quarter = warp & 3;
         const int sub = warp >= 8 ? 1 : 0;
         const int row = (quarter & 1) * 32 + lane;          // head row within this CTA
@@ -944,111 +953,141 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
         const uint32_t p_full_leader1 = map_to_rank(smem_u32(&ctl->p_full[1]), leader);
         float m_ref = -INFINITY, l = 0.f;
         bool ok = true;
-        for (int i = 0; i < tiles; ++i) {
-            const int buf = i & 1, sbuf = i % 3;
+        // Tiles alternate between two groups of four warps (2-5: even tiles, 8-11: odd tiles), so
+        // the chain scores -> weights of one tile overlaps the next tile's instead of all eight warps
+        // marching through every tile together.  In its group a thread serves head row `row` and
+        // the token half `half` of the tile (32 tokens, all 32 score columns of its lane).  The
+        // running reference maximum of a row is shared by the groups through ctl->ref: tile i reads
+        // what tile i-1 left and publishes its own decision at once, before its exponentials.
+        const int grp = sub;
+        for (int i = grp; ok && i < tiles; i += 2) {
+            const int sbuf = i % 3, it = i >> 1;
             ok = mbar_wait(&ctl->s_full[sbuf], (i / 3) & 1);
             if (!__all_sync(0xffffffffu, ok)) {
                 ok = false;
                 break;
             }
             tc_fence_after();
-            uint32_t sv[16];
-            tc_ld16(tmem + lane_base + kC2ColS + 32 * sbuf + 16 * sub, sv);
+            uint32_t sv[32];
+            tc_ld32(tmem + lane_base + kC2ColS + 32 * sbuf, sv);
             tc_wait_ld();
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(s_empty_leader + 8 * sbuf);
-            const uint32_t valid = (uint32_t)(ctl->valid_mask[i % kMaskRing] >> (16 * part)) & 0xffffu;
-            float x[16];
+            const uint32_t valid = (uint32_t)(ctl->valid_mask[i % kMaskRing] >> (32 * half));
+            float x[32];
             float mt = -INFINITY;
-            if (valid == 0xffffu) {
+            if (valid == 0xffffffffu) {
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
+                for (int j = 0; j < 32; ++j) {
                     x[j] = __uint_as_float(sv[j]) * p.scale_log2;
                     mt = fmaxf(mt, x[j]);
                 }
             } else {
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
+                for (int j = 0; j < 32; ++j) {
                     x[j] = ((valid >> j) & 1u) ? __uint_as_float(sv[j]) * p.scale_log2 : -INFINITY;
                     mt = fmaxf(mt, x[j]);
                 }
             }
-            ctl->xchg[i & 1][part][row] = mt;
-            mbar_arrive(&ctl->x_bar);
-            ok = mbar_wait(&ctl->x_bar, i & 1);
+            // the row's other half is served by the thread of the same lane two warps on
+            float *xg = &ctl->xchg[0][0][0] + ((grp * 2 + (it & 1)) * 2) * 64;      // [group][parity][half][row]
+            xg[half * 64 + row] = mt;
+            mbar_arrive(&ctl->xg_bar[grp]);
+            ok = mbar_wait(&ctl->xg_bar[grp], it & 1);
+            if (i > 0) ok = ok && mbar_wait(&ctl->ref_bar, (i - 1) & 1);
             if (!__all_sync(0xffffffffu, ok)) {
                 ok = false;
                 break;
             }
-            mt = fmaxf(fmaxf(ctl->xchg[i & 1][0][row], ctl->xchg[i & 1][1][row]),
-                       fmaxf(ctl->xchg[i & 1][2][row], ctl->xchg[i & 1][3][row]));
+            mt = fmaxf(mt, xg[(half ^ 1) * 64 + row]);
+            const float ref_in = i > 0 ? ctl->ref[(i - 1) & 1][row] : -INFINITY;
             // move the reference only when the tile maximum leaves the window above it
-            float factor = 1.f;
+            float ref_out = ref_in;
             bool moved = false;
-            if (mt > m_ref + kRescaleThreshold || (m_ref == -INFINITY && mt > -INFINITY)) {
-                factor = exp2f(m_ref - mt);
-                m_ref = mt;
+            if (mt > ref_in + kRescaleThreshold || (ref_in == -INFINITY && mt > -INFINITY)) {
+                ref_out = mt;
                 moved = true;
+            }
+            if (half == 0) ctl->ref[i & 1][row] = ref_out;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&ctl->ref_bar);
+            // this thread's own sum was last brought to reference m_ref
+            if (ref_out != m_ref) {
+                l *= (m_ref == -INFINITY) ? 0.f : exp2f(m_ref - ref_out);
+                m_ref = ref_out;
             }
             const float mr = (m_ref == -INFINITY) ? 0.f : m_ref;
             float sum = 0.f;
-            uint32_t pk[8];
+            uint32_t pk[16];
 #pragma unroll
-            for (int j = 0; j < 16; j += 2) {
+            for (int j = 0; j < 32; j += 2) {
                 const float e0 = exp2f(x[j] - mr), e1 = exp2f(x[j + 1] - mr);
                 sum += e0 + e1;
                 pk[j >> 1] = pack_bf16(e0, e1);
             }
-            l = l * factor + sum;
-            // the P buffer is free once P V of tile i-2 retired; O may be rescaled once P V of tile i-1 did
+            l += sum;
+            // this group's P buffer is free once P V of tile i-2 retired; O may be rescaled once P V of tile i-1 did
             if (i >= 2) {
-                ok = mbar_wait(&ctl->pv_done[buf], ((i >> 1) - 1) & 1);
+                ok = mbar_wait(&ctl->pv_done[grp], ((i >> 1) - 1) & 1);
                 if (!__all_sync(0xffffffffu, ok)) {
                     ok = false;
                     break;
                 }
             }
             if (i >= 1 && __any_sync(0xffffffffu, moved)) {
-                ok = mbar_wait(&ctl->pv_done[buf ^ 1], ((i - 1) >> 1) & 1);
+                ok = mbar_wait(&ctl->pv_done[grp ^ 1], ((i - 1) >> 1) & 1);
                 if (!__all_sync(0xffffffffu, ok)) {
                     ok = false;
                     break;
                 }
                 tc_fence_after();
+                // the four warps of the group cover all 128 lanes: each thread rescales the 256 value columns of its lane
+                const float factor = moved ? ((ref_in == -INFINITY) ? 0.f : exp2f(ref_in - ref_out)) : 1.f;
 #pragma unroll 1
-                for (int c = 0; c < 128; c += 32) {
+                for (int c = 0; c < 256; c += 32) {
                     uint32_t ov[32];
-                    tc_ld32(tmem + lane_base + kColO + 128 * sub + c, ov);
+                    tc_ld32(tmem + lane_base + kColO + c, ov);
                     tc_wait_ld();
 #pragma unroll
                     for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * factor);
-                    tc_st32(tmem + lane_base + kColO + 128 * sub + c, ov);
+                    tc_st32(tmem + lane_base + kColO + c, ov);
                 }
                 tc_wait_st();
             }
-            // P row quarter: 16 tokens x bf16 = two 16-byte chunks, chunk c stored at c ^ (row % 8)
-            uint8_t *p_row = smem + kC2SmemP + buf * kPanelBytes + row * 128;
+            // half a P row: 32 tokens x bf16 = four 16-byte chunks, chunk c stored at c ^ (row % 8)
+            uint8_t *p_row = smem + kC2SmemP + grp * kPanelBytes + row * 128;
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                const int chunk = (part * 2 + c) ^ (row & 7);
+            for (int c = 0; c < 4; ++c) {
+                const int chunk = (half * 4 + c) ^ (row & 7);
                 *reinterpret_cast<uint4 *>(p_row + chunk * 16) =
                     make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
             }
             fence_async_smem();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(buf ? p_full_leader1 : p_full_leader0);
+            if (lane == 0) mbar_arrive_cluster(grp ? p_full_leader1 : p_full_leader0);
         }
         if (ok) {
-            ok = mbar_wait(&ctl->pv_done[(tiles - 1) & 1], ((tiles - 1) >> 1) & 1);
+            // the last tile's P V has retired and its reference is the final one
+            ok = mbar_wait(&ctl->pv_done[(tiles - 1) & 1], ((tiles - 1) >> 1) & 1) && mbar_wait(&ctl->ref_bar, (tiles - 1) & 1);
             ok = __all_sync(0xffffffffu, ok);
         }
         if (ok) {
-            // total row sum: add the partial sums of the row's other three threads
-            ctl->xchg[tiles & 1][part][row] = l;
+            const float ref_final = ctl->ref[(tiles - 1) & 1][row];
+            if (ref_final != m_ref) {
+                l *= (m_ref == -INFINITY) ? 0.f : exp2f(m_ref - ref_final);
+                m_ref = ref_final;
+            }
+        }
+        constexpr int xs = 0;                                  // exchange slot of the final row sums
+        if (ok) {
+            // total row sum: add the partial sums of the row's other three threads (the groups'
+            // exchange slots are dead by now: the last P V could only be issued after every warp of
+            // its group had read its partner's maximum and written its weights)
+            ctl->xchg[xs][part][row] = l;
             mbar_arrive(&ctl->x_bar);
-            ok = mbar_wait(&ctl->x_bar, tiles & 1);
+            ok = mbar_wait(&ctl->x_bar, 0);
             ok = __all_sync(0xffffffffu, ok);
         }
         if (ok && p.cluster_merge) {
@@ -1057,14 +1096,12 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
             if (warp == 2 && lane == 0) mbar_arrive_cluster(map_to_rank(smem_u32(&ctl->ready_bar), crank ^ 2u));
             // the result stays in tensor memory: the exchange after the main loop normalises it and
             // hands half of it to the CTA that serves the same heads in the other split
-            const float lt = (ctl->xchg[tiles & 1][0][row] + ctl->xchg[tiles & 1][1][row]) +
-                             (ctl->xchg[tiles & 1][2][row] + ctl->xchg[tiles & 1][3][row]);
+            const float lt = (ctl->xchg[xs][0][row] + ctl->xchg[xs][1][row]) + (ctl->xchg[xs][2][row] + ctl->xchg[xs][3][row]);
             cm_inv = lt > 0.f ? 1.f / lt : 0.f;
             cm_lse = lt > 0.f ? (m_ref + log2f(lt)) * kLn2 : -INFINITY;
         } else if (ok) {
             tc_fence_after();
-            const float lt = (ctl->xchg[tiles & 1][0][row] + ctl->xchg[tiles & 1][1][row]) +
-                             (ctl->xchg[tiles & 1][2][row] + ctl->xchg[tiles & 1][3][row]);
+            const float lt = (ctl->xchg[xs][0][row] + ctl->xchg[xs][1][row]) + (ctl->xchg[xs][2][row] + ctl->xchg[xs][3][row]);
             c2_store_result(p, smem, tmem, warp, lane, b, s, h0, head_rows, lt, m_ref);
             const bool final_out = p.splits == 1;
             // with the in-kernel merge the partial results must be visible before this CTA is counted

@@ -85,7 +85,6 @@ struct Q8Control {
     uint64_t ready_bar;
     uint64_t valid_mask[kMaskRing];
     float xchg[2][4][64];
-    float xlse[2][64];
     uint32_t tmem_base;
     uint32_t abort;
     uint32_t merge_flag;
