@@ -841,11 +841,12 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
             // with thread-dependent control flow every MMA costs ~70 clocks to issue instead of ~25.
             const int tiles_u = __shfl_sync(0xffffffffu, tiles, 0);
             const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem, 0);
-            // The buffer parity is a compile-time constant of each issue routine (the tile loop is
-            // unrolled by two), so every operand of an MMA is a loop-invariant uniform value.
-            // S(t) = Q K(t)^T: 36 k-steps, Q panel c (8 KiB apart) against K panel c (4 KiB apart)
-            auto issue_qk = [&](auto kpar_tag, auto sbuf_tag) {
-                constexpr int kpar = decltype(kpar_tag)::value, sbuf = decltype(sbuf_tag)::value;
+            // One copy of each issue routine: stage and buffer enter as warp-uniform run-time values
+            // (every operand of an MMA is then a uniform base plus a compile-time offset), which
+            // keeps the issuing warp's code a few kilobytes instead of several tens (an issue loop
+            // unrolled over the buffer parities ran config-2-sized launches 5 % slower, token-level
+            // ones 8 %: a launch starts with cold instruction caches and this loop is its critical path).
+            auto issue_qk = [&](int kpar, int sbuf) {
                 const uint32_t d = tmem_u + kC2ColS + 32 * sbuf;
                 const uint32_t kb = k_lo + ((kpar * kC2KBytes) >> 4);
                 tc_mma_pair_elect<false>(d, q_lo, kmaj_hi, kb, kmaj_hi, idesc_qk);
@@ -856,9 +857,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
                 tc_commit_pair_elect(&ctl->k_empty[kpar], pair_mask);
                 tc_commit_pair_elect(&ctl->s_full[sbuf], pair_mask);
             };
-            // O += P(t) V(t): 4 k-steps of 16 tokens, two N=256 instructions each
-            auto issue_pv = [&](auto par_tag, bool first) {
-                constexpr int par = decltype(par_tag)::value;
+            auto issue_pv = [&](int par, bool first) {
                 const uint32_t a = p_lo + ((par * kPanelBytes) >> 4);
                 const uint32_t bd = v_lo + ((par * kC2VBytes) >> 4);
                 if (first) {
@@ -876,59 +875,45 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
                 }
                 tc_commit_pair_elect(&ctl->pv_done[par], pair_mask);
             };
-            // Q K^T runs two tiles ahead of P V (three S buffers), so the chain S ready -> softmax ->
-            // P -> P V of a tile has two tile times to complete before the tensor pipe needs it.
-            // S(t) lives in buffer t % 3, K(t) in stage t & 1.
-            auto qk_tile = [&](auto kpar_tag, auto sbuf_tag, int t) -> bool {
-                constexpr int kpar = decltype(kpar_tag)::value, sbuf = decltype(sbuf_tag)::value;
+            // S(t) lives in buffer t % 3, K(t) in stage t & 1; Q K^T runs two tiles ahead of P V
+            auto qk_tile = [&](int t) -> bool {
+                const int kpar = t & 1, sbuf = t % 3;
                 bool good = mbar_wait(&ctl->k_full[kpar], (t >> 1) & 1) &&
                             (t < 3 || mbar_wait(&ctl->s_empty[sbuf], ((t / 3) - 1) & 1));
                 good = __all_sync(0xffffffffu, good);
                 if (!good) return false;
                 tc_fence_after();
-                issue_qk(kpar_tag, sbuf_tag);
+                issue_qk(kpar, sbuf);
                 return true;
             };
-            auto pv_tile = [&](auto par_tag, int i) -> bool {
-                constexpr int par = decltype(par_tag)::value;
+            auto pv_tile = [&](int i) -> bool {
+                const int par = i & 1;
                 bool good = mbar_wait(&ctl->p_full[par], (i >> 1) & 1) && mbar_wait(&ctl->v_full[par], (i >> 1) & 1);
                 good = __all_sync(0xffffffffu, good);
                 if (!good) return false;
                 tc_fence_after();
-                issue_pv(par_tag, i == 0);
+                issue_pv(par, i == 0);
                 return true;
             };
-            using I0 = std::integral_constant<int, 0>;
-            using I1 = std::integral_constant<int, 1>;
-            using I2 = std::integral_constant<int, 2>;
-            // step j of a group of six tiles: Q K^T of tile i+2 (stage i & 1, buffer (i+2) % 3), then P V of tile i
-            // (if the K rows of tile i+2 have not landed yet while P and V of tile i are ready, P V goes first)
-            auto step = [&](auto kpar_tag, auto sbuf_tag, int i) -> bool {
-                constexpr int kpar = decltype(kpar_tag)::value;
+            bool ok = mbar_wait(&ctl->q_full, 0);
+            ok = __all_sync(0xffffffffu, ok);
+            if (ok) ok = qk_tile(0);
+            if (ok && tiles_u > 1) ok = qk_tile(1);
+            for (int i = 0; ok && i < tiles_u; ++i) {
+                // if the K rows of tile i+2 have not landed yet while P and V of tile i are ready, P V goes first
                 bool qk_todo = i + 2 < tiles_u;
                 if (qk_todo) {
+                    const int kpar = i & 1;
                     const bool k_ready = __all_sync(0xffffffffu, mbar_test(&ctl->k_full[kpar], ((i + 2) >> 1) & 1));
                     const bool pv_ready = __all_sync(0xffffffffu, mbar_test(&ctl->p_full[kpar], (i >> 1) & 1) &&
                                                                       mbar_test(&ctl->v_full[kpar], (i >> 1) & 1));
                     if (k_ready || !pv_ready) {
-                        if (!qk_tile(kpar_tag, sbuf_tag, i + 2)) return false;
+                        ok = qk_tile(i + 2);
                         qk_todo = false;
                     }
                 }
-                if (!pv_tile(kpar_tag, i)) return false;
-                return !qk_todo || qk_tile(kpar_tag, sbuf_tag, i + 2);
-            };
-            bool ok = mbar_wait(&ctl->q_full, 0);
-            ok = __all_sync(0xffffffffu, ok);
-            if (ok) ok = qk_tile(I0{}, I0{}, 0);
-            if (ok && tiles_u > 1) ok = qk_tile(I1{}, I1{}, 1);
-            for (int i = 0; ok && i < tiles_u; i += 6) {
-                ok = step(I0{}, I2{}, i);
-                if (ok && i + 1 < tiles_u) ok = step(I1{}, I0{}, i + 1);
-                if (ok && i + 2 < tiles_u) ok = step(I0{}, I1{}, i + 2);
-                if (ok && i + 3 < tiles_u) ok = step(I1{}, I2{}, i + 3);
-                if (ok && i + 4 < tiles_u) ok = step(I0{}, I0{}, i + 4);
-                if (ok && i + 5 < tiles_u) ok = step(I1{}, I1{}, i + 5);
+                if (ok) ok = pv_tile(i);
+                if (ok && qk_todo) ok = qk_tile(i + 2);
             }
             if (!ok && lane == 0) {
                 flag_status(p.status, OMNI_DEV_TIMEOUT | OMNI_DEV_ROLE_MMA);

@@ -93,8 +93,7 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes)
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, long long limit = kWaitCycles)
 {
     const uint32_t addr = smem_u32(bar);
-    const long long start = clock64();
-    for (uint32_t it = 0;; ++it) {
+    auto attempt = [&]() {
         uint32_t done;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
@@ -103,7 +102,14 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, long l
             : "=r"(done)
             : "r"(addr), "r"(parity)
             : "memory");
-        if (done) return true;
+        return done != 0;
+    };
+    // the clock is only read once the first attempt has failed: most waits of the pipeline find
+    // their phase complete or completing, and they sit on its critical path
+    if (attempt()) return true;
+    const long long start = clock64();
+    for (uint32_t it = 0;; ++it) {
+        if (attempt()) return true;
         if ((it & 63u) == 63u && clock64() - start > limit) return false;
     }
 }
