@@ -117,7 +117,15 @@ def oracle_subset_q8(w, cache, scale, reqs=None, heads=None):
     sl = w.sel_len.cpu().numpy()[reqs]
     rows = oracle.resolve_rows(pt, si, sl, w.page_size, w.num_pages)
     gather = torch.from_numpy(np.where(rows < 0, 0, rows)).to(cache.device).view(-1)
-    krows = q8.dequantise_rows(cache[gather].cpu().numpy(), scale[gather].cpu().numpy()).reshape(len(reqs), -1, w.d_qk)
+    # the rows the oracle attends to are quantised by the oracle itself from the seeded bf16 pool;
+    # the device-made cache must hold the same bits there, and is not otherwise used as an input
+    bits = w.kv_cache.view(-1, w.d_qk)[gather].cpu().view(torch.int16).numpy().view(np.uint16)
+    own_cache, own_scale = q8.quantise_rows(bits)
+    live = np.asarray(rows).reshape(-1) >= 0
+    assert np.array_equal(cache[gather].cpu().numpy()[live], own_cache[live]), "codes of the selected rows differ"
+    assert np.array_equal(scale[gather].cpu().numpy().view(np.uint32)[live], own_scale.view(np.uint32)[live]), \
+        "scales of the selected rows differ"
+    krows = q8.dequantise_rows(own_cache, own_scale).reshape(len(reqs), -1, w.d_qk)
     q = w.q[torch.tensor(reqs, device=w.q.device)][:, torch.tensor(heads, device=w.q.device)].cpu().to(torch.float64).numpy()
     return q8.attend_dequantised(q, krows, sl, w.d_v, w.scale)
 
