@@ -256,13 +256,16 @@ __device__ __forceinline__ void tc_commit_pair_elect(uint64_t *bar, uint16_t bot
 // Split-KV merge inside a cluster of two pairs, i.e. the two splits of one request (cluster
 // merge).  CTA `crank` and its partner `crank ^ 2` serve the same 64 heads in the two splits.
 // Instead of writing fp32 partial results to global memory for a second kernel to read back,
-// the two exchange what the other needs through distributed shared memory:
-//   1. each normalises its accumulator by its row sums, keeps the 256 value columns it will
-//      finish (split 0: columns 0..255, split 1: 256..511) and sends the other 256, followed by
-//      the log-sum-exp of its split for every head row, to the partner with one bulk
-//      shared-memory-to-shared-memory copy;
-//   2. each weighs what it kept and what it received by exp(lse_split - lse_total), adds them
-//      and stores its half of the final rows.
+// the two exchange what the other needs through distributed shared memory.  Of every head row
+// split 0 finishes value columns [0,128) and [256,384), split 1 the other two quarters: these are
+// the columns of softmax warps 2-5 and 8-11 in tensor memory, so in either CTA one warp per
+// scheduler is a "sender" (its columns are finished by the partner) and one a "keeper":
+//   1. the senders normalise their half by the row sums and write it, followed by the
+//      log-sum-exp of the split for every head row, to one block of shared memory, which one bulk
+//      shared-memory-to-shared-memory copy takes to the partner;
+//   2. the keepers wait for the partner's block, weigh their own half (still in tensor memory)
+//      and the received one by exp(lse_split - lse_total), add them and store bf16 rows as whole
+//      128-byte lines through warp-private staging tiles.
 // The copy lands in shared memory that held the partner's operand tiles, so it is not sent
 // before the partner has said that its main loop is over (`ready_bar`, a remote arrive that the
 // partner fires as soon as its last P V has retired, while this CTA is still staging).
@@ -276,112 +279,146 @@ __device__ __forceinline__ void cluster_merge_exchange(const DecodeParams &p, Co
     constexpr uint32_t kPitch = kSliceBytes + 16;        // row-per-lane 16-byte accesses do not conflict
     constexpr uint32_t kRowsBytes = 64 * kPitch;         // 66,560
     constexpr uint32_t kBlockBytes = kRowsBytes + 256;   // + 64 log-sum-exps
-    static_assert(3 * kBlockBytes + 512 <= kC2SmemCtl, "exchange tiles must fit below the control block");
-    uint8_t *send = smem, *keep = smem + kBlockBytes, *recv = smem + 2 * kBlockBytes;
-    float(*xlse)[64] = reinterpret_cast<float(*)[64]>(smem + 3 * kBlockBytes);   // weights of the two splits per head row
+    constexpr uint32_t kStagePitch = 144, kStageBytes = 32 * kStagePitch;
+    static_assert(3 * kBlockBytes <= kC2SmemCtl, "exchange tiles must fit below the control block");
+    static_assert(8 * kStageBytes <= kBlockBytes, "four warps' staging tiles sit between the two blocks");
+    uint8_t *send = smem, *stages = smem + kBlockBytes, *recv = smem + 2 * kBlockBytes;
     const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;
     const bool is_softmax = (warp >= 2 && warp <= 5) || warp >= 8;
     if (!is_softmax) return;
     const int quarter = warp & 3, sub = warp >= 8 ? 1 : 0;
-    const int row = (quarter & 1) * 32 + lane, part = (quarter >> 1) * 2 + sub;
+    const int row = (quarter & 1) * 32 + lane, half = quarter >> 1;
     const uint32_t partner = crank ^ 2u;
-    // an empty split never ran a main loop: its shared memory is free from the start
-    if (!active && warp == 2 && lane == 0) mbar_arrive_cluster(map_to_rank(smem_u32(&ctl->ready_bar), partner));
-    // Whether anything went wrong is decided for the whole CTA, never per warp: all eight warps
-    // pass the same named barriers below and then go on or leave together.  A warp whose main
-    // loop ran into a bounded wait says so here; the decision is read after the next barrier.
+    const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
     volatile uint32_t *xfail = &ctl->xfail;
     if (!main_ok && lane == 0) *xfail = 1u;
+    // The partner may overwrite this CTA's operand tiles once it has been told that the main loop
+    // here is over.  Warp 2 says so at the end of a main loop that went well; after one that did
+    // not (or that never ran: an empty split) the same thread says so here, so that the arrive is
+    // fired exactly once per launch whatever happened.
+    if (warp == 2 && lane == 0 && (!active || !main_ok)) mbar_arrive_cluster(map_to_rank(smem_u32(&ctl->ready_bar), partner));
 
-    // this thread's 128 value columns are finished by split `part / 2`
-    uint8_t *tile = ((part >> 1) == s ? keep : send) + (size_t)row * kPitch + (part & 1) * 512;
-    const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+    // No warp leaves this function early and no barrier below depends on how a wait ended: the
+    // four sending warps always meet at their named barrier, every wait is bounded, and a wait
+    // that ran out only marks the launch as failed (its results are then unspecified).
+    tc_fence_after();
+    if (sub != s) {
+        // ---- sender: this thread's 128 value columns are finished by the other split ----------
+        uint8_t *tile = send + (size_t)row * kPitch + half * 512;
 #pragma unroll 1
-    for (int q = 0; q < 4; ++q) {
-        uint32_t ov[32];
-        __syncwarp();
-        if (active) {
-            tc_ld32(tmem + lane_base + kColO + 128 * sub + q * 32, ov);
-            tc_wait_ld();
-        }
-        uint4 *o = reinterpret_cast<uint4 *>(tile + q * 128);
+        for (int q = 0; q < 4; ++q) {
+            uint32_t ov[32];
+            __syncwarp();
+            if (active) {
+                tc_ld32(tmem + lane_base + kColO + 128 * sub + q * 32, ov);
+                tc_wait_ld();
+            }
+            uint4 *o = reinterpret_cast<uint4 *>(tile + q * 128);
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            // an empty or fully masked split contributes exact zeros
-            o[j] = (active && cm_inv != 0.f)
-                       ? make_uint4(__float_as_uint(__uint_as_float(ov[4 * j]) * cm_inv),
-                                    __float_as_uint(__uint_as_float(ov[4 * j + 1]) * cm_inv),
-                                    __float_as_uint(__uint_as_float(ov[4 * j + 2]) * cm_inv),
-                                    __float_as_uint(__uint_as_float(ov[4 * j + 3]) * cm_inv))
-                       : make_uint4(0u, 0u, 0u, 0u);
+            for (int j = 0; j < 8; ++j) {
+                // an empty or fully masked split contributes exact zeros
+                o[j] = (active && cm_inv != 0.f)
+                           ? make_uint4(__float_as_uint(__uint_as_float(ov[4 * j]) * cm_inv),
+                                        __float_as_uint(__uint_as_float(ov[4 * j + 1]) * cm_inv),
+                                        __float_as_uint(__uint_as_float(ov[4 * j + 2]) * cm_inv),
+                                        __float_as_uint(__uint_as_float(ov[4 * j + 3]) * cm_inv))
+                           : make_uint4(0u, 0u, 0u, 0u);
+            }
         }
-    }
-    if (part == 0) reinterpret_cast<float *>(send + kRowsBytes)[row] = cm_lse;
-    tc_fence_before();
-    fence_async_smem();                                   // the bulk copy reads what the threads wrote
-    asm volatile("bar.sync 1, 256;" ::: "memory");         // the eight softmax warps
-    const bool main_failed = *xfail != 0u;
-    if (warp == 2) {
-        // A CTA whose main loop gave up never told its partner that its operand tiles are dead
-        // (that arrive sits at the end of the main loop).  It does so now, and it still sends a
-        // block (of unspecified contents: the status word already says so), so that every wait
-        // of the healthy partner ends and both CTAs finish together.
-        if (main_failed && active && lane == 0) mbar_arrive_cluster(map_to_rank(smem_u32(&ctl->ready_bar), partner));
-        bool ready = mbar_wait(&ctl->ready_bar, 0);       // the partner's operand tiles are dead
-        ready = __all_sync(0xffffffffu, ready);
-        if (ready && lane == 0) {
-            mbar_expect_tx(&ctl->recv_bar, kBlockBytes);
-            const uint32_t dst = map_to_rank(smem_u32(recv), partner);
-            const uint32_t bar = map_to_rank(smem_u32(&ctl->recv_bar), partner);
-            asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                         ::"r"(dst), "r"(smem_u32(send)), "r"(kBlockBytes), "r"(bar)
-                         : "memory");
+        if (half == 0) reinterpret_cast<float *>(send + kRowsBytes)[row] = cm_lse;
+        tc_fence_before();
+        fence_async_smem();                               // the bulk copy reads what the threads wrote
+        asm volatile("bar.sync 2, 128;" ::: "memory");     // the four sending warps
+        if (quarter == 0) {
+            bool ready = mbar_wait(&ctl->ready_bar, 0);   // the partner's operand tiles are dead
+            ready = __all_sync(0xffffffffu, ready);
+            if (ready && lane == 0) {
+                const uint32_t dst = map_to_rank(smem_u32(recv), partner);
+                const uint32_t bar = map_to_rank(smem_u32(&ctl->recv_bar), partner);
+                asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                             ::"r"(dst), "r"(smem_u32(send)), "r"(kBlockBytes), "r"(bar)
+                             : "memory");
+            }
+            if (!ready && lane == 0) {
+                *xfail = 1u;
+                flag_status(p.status, OMNI_DEV_TIMEOUT | OMNI_DEV_ROLE_SOFTMAX);
+            }
         }
-        if (!ready && lane == 0) *xfail = 1u;
+        return;
     }
+
+    // ---- keeper: this thread's 128 value columns are finished here -----------------------------
+    // The kept half never leaves tensor memory: once the partner's block is in, each thread mixes
+    // its own accumulator row with the received one, 64 columns a round, and the warp writes the
+    // bf16 rows out as whole 128-byte lines through its private staging tile.
+    if (quarter == 0 && lane == 0) mbar_expect_tx(&ctl->recv_bar, kBlockBytes);
     {
         bool got = mbar_wait(&ctl->recv_bar, 0);
         got = __all_sync(0xffffffffu, got);
-        if (!got && lane == 0) *xfail = 1u;
-    }
-    asm volatile("bar.sync 1, 256;" ::: "memory");         // every warp's verdict is in
-    if (*xfail != 0u) {
-        if (warp == 2 && lane == 0) flag_status(p.status, OMNI_DEV_TIMEOUT | OMNI_DEV_ROLE_SOFTMAX);
-        return;                                            // all eight warps leave here together
-    }
-    // weights of the two splits per head row (in place of the log-sum-exps), final log-sum-exp
-    if (part == 0) {
-        const float other = reinterpret_cast<const float *>(recv + kRowsBytes)[row];
-        const float mx = fmaxf(cm_lse, other);
-        float total = -INFINITY, w_own = 0.f, w_other = 0.f;
-        if (mx > -INFINITY) {
-            total = mx + logf(exp2f((cm_lse - mx) * kLog2e) + exp2f((other - mx) * kLog2e));
-            if (cm_lse > -INFINITY) w_own = exp2f((cm_lse - total) * kLog2e);
-            if (other > -INFINITY) w_other = exp2f((other - total) * kLog2e);
+        if (!got && lane == 0) {
+            *xfail = 1u;
+            flag_status(p.status, OMNI_DEV_TIMEOUT | OMNI_DEV_ROLE_SOFTMAX);
         }
-        xlse[0][row] = w_own;
-        xlse[1][row] = w_other;
-        if (s == 0 && row < head_rows) p.lse[(size_t)b * p.heads + h0 + row] = total;
     }
-    asm volatile("bar.sync 1, 256;" ::: "memory");
-    // kept + received -> bf16, 16 output bytes (8 columns) per item, consecutive threads along a row
-    const int t = (sub * 4 + ((warp - 2) & 3)) * 32 + lane;          // 0..255
-    for (int item = t; item < head_rows * 32; item += 256) {
-        const int r = item >> 5, c = item & 31;
-        const float wk = xlse[0][r], wr = xlse[1][r];
-        const uint4 *k4 = reinterpret_cast<const uint4 *>(keep + (size_t)r * kPitch + c * 32);
-        const uint4 *r4 = reinterpret_cast<const uint4 *>(recv + (size_t)r * kPitch + c * 32);
-        const uint4 k0 = k4[0], k1 = k4[1], r0 = r4[0], r1 = r4[1];
-        // a weight of zero must not meet a non-finite partner value
-        auto mix = [&](uint32_t kv, uint32_t rv) {
-            return (wk != 0.f ? wk * __uint_as_float(kv) : 0.f) + (wr != 0.f ? wr * __uint_as_float(rv) : 0.f);
-        };
-        uint4 o;
-        o.x = pack_bf16(mix(k0.x, r0.x), mix(k0.y, r0.y));
-        o.y = pack_bf16(mix(k0.z, r0.z), mix(k0.w, r0.w));
-        o.z = pack_bf16(mix(k1.x, r1.x), mix(k1.y, r1.y));
-        o.w = pack_bf16(mix(k1.z, r1.z), mix(k1.w, r1.w));
-        *reinterpret_cast<uint4 *>(p.out + ((size_t)b * p.heads + h0 + r) * kDv + s * 256 + c * 8) = o;
+    // weights of the two splits for this head row, final log-sum-exp
+    const float other = reinterpret_cast<const float *>(recv + kRowsBytes)[row];
+    const float mx = fmaxf(cm_lse, other);
+    float total = -INFINITY, w_own = 0.f, w_other = 0.f;
+    if (mx > -INFINITY) {
+        total = mx + logf(exp2f((cm_lse - mx) * kLog2e) + exp2f((other - mx) * kLog2e));
+        if (cm_lse > -INFINITY) w_own = exp2f((cm_lse - total) * kLog2e);
+        if (other > -INFINITY) w_other = exp2f((other - total) * kLog2e);
+    }
+    if (s == 0 && half == 0 && row < head_rows) p.lse[(size_t)b * p.heads + h0 + row] = total;
+    // An accumulator that carries no weight is not read at all (that of an empty split was never
+    // written, that of a fully masked one may hold anything); the partner sends exact zeros then.
+    const bool use_own = active && cm_inv != 0.f && w_own != 0.f;
+    const float f_own = use_own ? w_own * cm_inv : 0.f, f_other = w_other;
+    const int widx = quarter;                                             // 0..3 among the keeping warps
+    uint8_t *stage = stages + (size_t)widx * 2 * kStageBytes;
+    const int row0 = (quarter & 1) * 32;                                  // first head row of this warp
+    uint8_t *gbase = reinterpret_cast<uint8_t *>(p.out + ((size_t)b * p.heads + h0 + row0) * kDv + half * 256 + sub * 128);
+    const int rows_here = max(0, min(32, head_rows - row0));
+    const uint8_t *theirs = recv + (size_t)row * kPitch + half * 512;
+#pragma unroll 1
+    for (int q = 0; q < 2; ++q) {
+        uint8_t *buf = stage + (q & 1) * kStageBytes;
+        uint4 *mine = reinterpret_cast<uint4 *>(buf + lane * kStagePitch);
+        __syncwarp();
+#pragma unroll
+        for (int c2 = 0; c2 < 2; ++c2) {
+            uint32_t ov[32];
+            if (use_own) {
+                tc_ld32(tmem + lane_base + kColO + 128 * sub + q * 64 + c2 * 32, ov);
+                tc_wait_ld();
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) ov[j] = 0u;
+            }
+            const uint4 *r4 = reinterpret_cast<const uint4 *>(theirs + q * 256 + c2 * 128);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint4 ra = r4[2 * j], rb = r4[2 * j + 1];
+                auto mix = [&](uint32_t own, uint32_t got) { return fmaf(f_own, __uint_as_float(own), f_other * __uint_as_float(got)); };
+                uint4 w;
+                w.x = pack_bf16(mix(ov[8 * j], ra.x), mix(ov[8 * j + 1], ra.y));
+                w.y = pack_bf16(mix(ov[8 * j + 2], ra.z), mix(ov[8 * j + 3], ra.w));
+                w.z = pack_bf16(mix(ov[8 * j + 4], rb.x), mix(ov[8 * j + 5], rb.y));
+                w.w = pack_bf16(mix(ov[8 * j + 6], rb.z), mix(ov[8 * j + 7], rb.w));
+                mine[c2 * 4 + j] = w;
+            }
+        }
+        __syncwarp();
+        uint8_t *gq = gbase + q * 128;
+        uint4 v[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+            v[k] = *reinterpret_cast<const uint4 *>(buf + (4 * k + (lane >> 3)) * kStagePitch + (lane & 7) * 16);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const int r = 4 * k + (lane >> 3);
+            if (r < rows_here) *reinterpret_cast<uint4 *>(gq + (size_t)r * (kDv * 2) + (lane & 7) * 16) = v[k];
+        }
     }
 }
 
