@@ -344,14 +344,16 @@ __device__ __forceinline__ void cluster_merge_exchange(const DecodeParams &p, Co
                 flag_status(p.status, OMNI_DEV_TIMEOUT | OMNI_DEV_ROLE_SOFTMAX);
             }
         }
-        return;
+    } else if (quarter == 0 && lane == 0) {
+        mbar_expect_tx(&ctl->recv_bar, kBlockBytes);
     }
 
-    // ---- keeper: this thread's 128 value columns are finished here -----------------------------
-    // The kept half never leaves tensor memory: once the partner's block is in, each thread mixes
-    // its own accumulator row with the received one, 64 columns a round, and the warp writes the
+    // ---- finish: the columns kept here (those of the warps with sub == s) never left tensor
+    // memory.  Once the partner's block is in, all eight warps take part: a warp can read any
+    // column of its tensor-memory lane quarter, so the keeping warp of a quarter finishes the
+    // first 64 of its 128 columns and the sending warp of the same quarter, its block gone, the
+    // other 64.  A thread mixes its accumulator row with the received one and the warp writes the
     // bf16 rows out as whole 128-byte lines through its private staging tile.
-    if (quarter == 0 && lane == 0) mbar_expect_tx(&ctl->recv_bar, kBlockBytes);
     {
         bool got = mbar_wait(&ctl->recv_bar, 0);
         got = __all_sync(0xffffffffu, got);
@@ -369,56 +371,51 @@ __device__ __forceinline__ void cluster_merge_exchange(const DecodeParams &p, Co
         if (cm_lse > -INFINITY) w_own = exp2f((cm_lse - total) * kLog2e);
         if (other > -INFINITY) w_other = exp2f((other - total) * kLog2e);
     }
-    if (s == 0 && half == 0 && row < head_rows) p.lse[(size_t)b * p.heads + h0 + row] = total;
+    if (s == 0 && sub == 0 && half == 0 && row < head_rows) p.lse[(size_t)b * p.heads + h0 + row] = total;
     // An accumulator that carries no weight is not read at all (that of an empty split was never
     // written, that of a fully masked one may hold anything); the partner sends exact zeros then.
     const bool use_own = active && cm_inv != 0.f && w_own != 0.f;
     const float f_own = use_own ? w_own * cm_inv : 0.f, f_other = w_other;
-    const int widx = quarter;                                             // 0..3 among the keeping warps
-    uint8_t *stage = stages + (size_t)widx * 2 * kStageBytes;
+    const int col = 128 * s + (sub == s ? 0 : 64);                        // first of this thread's 64 columns within its half
+    uint8_t *buf = stages + (size_t)(sub * 4 + quarter) * kStageBytes;
     const int row0 = (quarter & 1) * 32;                                  // first head row of this warp
-    uint8_t *gbase = reinterpret_cast<uint8_t *>(p.out + ((size_t)b * p.heads + h0 + row0) * kDv + half * 256 + sub * 128);
+    uint8_t *gq = reinterpret_cast<uint8_t *>(p.out + ((size_t)b * p.heads + h0 + row0) * kDv + half * 256 + col);
     const int rows_here = max(0, min(32, head_rows - row0));
-    const uint8_t *theirs = recv + (size_t)row * kPitch + half * 512;
-#pragma unroll 1
-    for (int q = 0; q < 2; ++q) {
-        uint8_t *buf = stage + (q & 1) * kStageBytes;
-        uint4 *mine = reinterpret_cast<uint4 *>(buf + lane * kStagePitch);
-        __syncwarp();
+    const uint8_t *theirs = recv + (size_t)row * kPitch + half * 512 + (sub == s ? 0 : 256);
+    uint4 *mine = reinterpret_cast<uint4 *>(buf + lane * kStagePitch);
+    tc_fence_after();
 #pragma unroll
-        for (int c2 = 0; c2 < 2; ++c2) {
-            uint32_t ov[32];
-            if (use_own) {
-                tc_ld32(tmem + lane_base + kColO + 128 * sub + q * 64 + c2 * 32, ov);
-                tc_wait_ld();
-            } else {
+    for (int c2 = 0; c2 < 2; ++c2) {
+        uint32_t ov[32];
+        if (use_own) {
+            tc_ld32(tmem + lane_base + kColO + col + c2 * 32, ov);
+            tc_wait_ld();
+        } else {
 #pragma unroll
-                for (int j = 0; j < 32; ++j) ov[j] = 0u;
-            }
-            const uint4 *r4 = reinterpret_cast<const uint4 *>(theirs + q * 256 + c2 * 128);
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const uint4 ra = r4[2 * j], rb = r4[2 * j + 1];
-                auto mix = [&](uint32_t own, uint32_t got) { return fmaf(f_own, __uint_as_float(own), f_other * __uint_as_float(got)); };
-                uint4 w;
-                w.x = pack_bf16(mix(ov[8 * j], ra.x), mix(ov[8 * j + 1], ra.y));
-                w.y = pack_bf16(mix(ov[8 * j + 2], ra.z), mix(ov[8 * j + 3], ra.w));
-                w.z = pack_bf16(mix(ov[8 * j + 4], rb.x), mix(ov[8 * j + 5], rb.y));
-                w.w = pack_bf16(mix(ov[8 * j + 6], rb.z), mix(ov[8 * j + 7], rb.w));
-                mine[c2 * 4 + j] = w;
-            }
+            for (int j = 0; j < 32; ++j) ov[j] = 0u;
         }
-        __syncwarp();
-        uint8_t *gq = gbase + q * 128;
-        uint4 v[8];
+        const uint4 *r4 = reinterpret_cast<const uint4 *>(theirs + c2 * 128);
 #pragma unroll
-        for (int k = 0; k < 8; ++k)
-            v[k] = *reinterpret_cast<const uint4 *>(buf + (4 * k + (lane >> 3)) * kStagePitch + (lane & 7) * 16);
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            const int r = 4 * k + (lane >> 3);
-            if (r < rows_here) *reinterpret_cast<uint4 *>(gq + (size_t)r * (kDv * 2) + (lane & 7) * 16) = v[k];
+        for (int j = 0; j < 4; ++j) {
+            const uint4 ra = r4[2 * j], rb = r4[2 * j + 1];
+            auto mix = [&](uint32_t own, uint32_t got) { return fmaf(f_own, __uint_as_float(own), f_other * __uint_as_float(got)); };
+            uint4 w;
+            w.x = pack_bf16(mix(ov[8 * j], ra.x), mix(ov[8 * j + 1], ra.y));
+            w.y = pack_bf16(mix(ov[8 * j + 2], ra.z), mix(ov[8 * j + 3], ra.w));
+            w.z = pack_bf16(mix(ov[8 * j + 4], rb.x), mix(ov[8 * j + 5], rb.y));
+            w.w = pack_bf16(mix(ov[8 * j + 6], rb.z), mix(ov[8 * j + 7], rb.w));
+            mine[c2 * 4 + j] = w;
         }
+    }
+    __syncwarp();
+    uint4 v[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k)
+        v[k] = *reinterpret_cast<const uint4 *>(buf + (4 * k + (lane >> 3)) * kStagePitch + (lane & 7) * 16);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const int r = 4 * k + (lane >> 3);
+        if (r < rows_here) *reinterpret_cast<uint4 *>(gq + (size_t)r * (kDv * 2) + (lane & 7) * 16) = v[k];
     }
 }
 
