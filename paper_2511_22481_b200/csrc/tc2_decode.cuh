@@ -86,7 +86,7 @@ struct C2Control {
     uint64_t x_bar;                      // all softmax threads: exchange of the final row sums
     uint64_t exit_bar;                   // both CTAs of the pair are done with tensor memory
     uint64_t valid_mask[kMaskRing];      // per tile: validity of its 64 tokens
-    float xchg[2][4][64];                // row maxima: [group][parity of the group's tile][token half][head row]; at the end [0][thread of the row][head row]: row sums
+    float xchg[2][4][64];                // row maxima: [group][2 * parity of the group's tile + token half][head row]; at the end the slots a group no longer uses carry its partial row sums
     uint32_t tmem_base;
     uint32_t abort;
     uint32_t merge_flag;
@@ -261,8 +261,9 @@ __device__ __forceinline__ void tc_commit_pair_elect(uint64_t *bar, uint16_t bot
 // the columns of softmax warps 2-5 and 8-11 in tensor memory, so in either CTA one warp per
 // scheduler is a "sender" (its columns are finished by the partner) and one a "keeper":
 //   1. the senders normalise their half by the row sums and write it, followed by the
-//      log-sum-exp of the split for every head row, to one block of shared memory, which one bulk
-//      shared-memory-to-shared-memory copy takes to the partner;
+//      log-sum-exp of the split for every head row, to one block of shared memory, which four
+//      bulk shared-memory-to-shared-memory copies take to the partner, each as soon as its
+//      quarter of the block is written;
 //   2. the keepers wait for the partner's block, weigh their own half (still in tensor memory)
 //      and the received one by exp(lse_split - lse_total), add them and store bf16 rows as whole
 //      128-byte lines through warp-private staging tiles.
@@ -275,14 +276,15 @@ __device__ __forceinline__ void cluster_merge_exchange(const DecodeParams &p, Co
                                                        uint32_t tmem, int b, int s, uint32_t crank, int h0,
                                                        int head_rows, bool active, bool main_ok, float cm_lse, float cm_inv)
 {
-    constexpr uint32_t kSliceBytes = 256 * 4;            // half of a row's value columns, fp32
-    constexpr uint32_t kPitch = kSliceBytes + 16;        // row-per-lane 16-byte accesses do not conflict
-    constexpr uint32_t kRowsBytes = 64 * kPitch;         // 66,560
-    constexpr uint32_t kBlockBytes = kRowsBytes + 256;   // + 64 log-sum-exps
+    // The block travels as four chunks, so that the copy of one overlaps the staging of the next:
+    // chunk q holds, for every head row, the q-th 32 columns of both 128-column runs that are sent.
+    constexpr uint32_t kChunkPitch = 2 * 128 + 16;       // row-per-lane 16-byte accesses do not conflict
+    constexpr uint32_t kChunkBytes = 64 * kChunkPitch;   // 17,408
+    constexpr uint32_t kRowsBytes = 4 * kChunkBytes;
+    constexpr uint32_t kBlockBytes = kRowsBytes + 256;   // + 64 log-sum-exps: 69,888
     constexpr uint32_t kStagePitch = 144, kStageBytes = 32 * kStagePitch;
-    static_assert(3 * kBlockBytes <= kC2SmemCtl, "exchange tiles must fit below the control block");
-    static_assert(8 * kStageBytes <= kBlockBytes, "four warps' staging tiles sit between the two blocks");
-    uint8_t *send = smem, *stages = smem + kBlockBytes, *recv = smem + 2 * kBlockBytes;
+    static_assert(2 * kBlockBytes + 8 * kStageBytes <= 221184, "exchange tiles must end below the control block and the 8-bit kernel's auxiliary arrays");
+    uint8_t *send = smem, *stages = smem + kBlockBytes, *recv = smem + kBlockBytes + 8 * kStageBytes;
     const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;
     const bool is_softmax = (warp >= 2 && warp <= 5) || warp >= 8;
     if (!is_softmax) return;
@@ -304,7 +306,8 @@ __device__ __forceinline__ void cluster_merge_exchange(const DecodeParams &p, Co
     tc_fence_after();
     if (sub != s) {
         // ---- sender: this thread's 128 value columns are finished by the other split ----------
-        uint8_t *tile = send + (size_t)row * kPitch + half * 512;
+        if (half == 0) reinterpret_cast<float *>(send + kRowsBytes)[row] = cm_lse;
+        bool ready = true;                                // (sending warp) the partner's operand tiles are dead
 #pragma unroll 1
         for (int q = 0; q < 4; ++q) {
             uint32_t ov[32];
@@ -313,7 +316,7 @@ __device__ __forceinline__ void cluster_merge_exchange(const DecodeParams &p, Co
                 tc_ld32(tmem + lane_base + kColO + 128 * sub + q * 32, ov);
                 tc_wait_ld();
             }
-            uint4 *o = reinterpret_cast<uint4 *>(tile + q * 128);
+            uint4 *o = reinterpret_cast<uint4 *>(send + q * kChunkBytes + (size_t)row * kChunkPitch + half * 128);
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 // an empty or fully masked split contributes exact zeros
@@ -324,24 +327,25 @@ __device__ __forceinline__ void cluster_merge_exchange(const DecodeParams &p, Co
                                         __float_as_uint(__uint_as_float(ov[4 * j + 3]) * cm_inv))
                            : make_uint4(0u, 0u, 0u, 0u);
             }
-        }
-        if (half == 0) reinterpret_cast<float *>(send + kRowsBytes)[row] = cm_lse;
-        tc_fence_before();
-        fence_async_smem();                               // the bulk copy reads what the threads wrote
-        asm volatile("bar.sync 2, 128;" ::: "memory");     // the four sending warps
-        if (quarter == 0) {
-            bool ready = mbar_wait(&ctl->ready_bar, 0);   // the partner's operand tiles are dead
-            ready = __all_sync(0xffffffffu, ready);
-            if (ready && lane == 0) {
-                const uint32_t dst = map_to_rank(smem_u32(recv), partner);
-                const uint32_t bar = map_to_rank(smem_u32(&ctl->recv_bar), partner);
-                asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                             ::"r"(dst), "r"(smem_u32(send)), "r"(kBlockBytes), "r"(bar)
-                             : "memory");
-            }
-            if (!ready && lane == 0) {
-                *xfail = 1u;
-                flag_status(p.status, OMNI_DEV_TIMEOUT | OMNI_DEV_ROLE_SOFTMAX);
+            fence_async_smem();                           // the bulk copy reads what the threads wrote
+            asm volatile("bar.sync 2, 128;" ::: "memory"); // the four sending warps
+            if (quarter == 0) {
+                if (q == 0) {
+                    ready = mbar_wait(&ctl->ready_bar, 0);
+                    ready = __all_sync(0xffffffffu, ready);
+                    if (!ready && lane == 0) {
+                        *xfail = 1u;
+                        flag_status(p.status, OMNI_DEV_TIMEOUT | OMNI_DEV_ROLE_SOFTMAX);
+                    }
+                }
+                if (ready && lane == 0) {
+                    const uint32_t bytes = q == 3 ? kChunkBytes + 256 : kChunkBytes;       // the last one takes the log-sum-exps along
+                    const uint32_t dst = map_to_rank(smem_u32(recv + q * kChunkBytes), partner);
+                    const uint32_t bar = map_to_rank(smem_u32(&ctl->recv_bar), partner);
+                    asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                                 ::"r"(dst), "r"(smem_u32(send + q * kChunkBytes)), "r"(bytes), "r"(bar)
+                                 : "memory");
+                }
             }
         }
     } else if (quarter == 0 && lane == 0) {
@@ -381,7 +385,7 @@ __device__ __forceinline__ void cluster_merge_exchange(const DecodeParams &p, Co
     const int row0 = (quarter & 1) * 32;                                  // first head row of this warp
     uint8_t *gq = reinterpret_cast<uint8_t *>(p.out + ((size_t)b * p.heads + h0 + row0) * kDv + half * 256 + col);
     const int rows_here = max(0, min(32, head_rows - row0));
-    const uint8_t *theirs = recv + (size_t)row * kPitch + half * 512 + (sub == s ? 0 : 256);
+    const uint8_t *theirs = recv + (sub == s ? 0 : 2) * kChunkBytes + (size_t)row * kChunkPitch + half * 128;
     uint4 *mine = reinterpret_cast<uint4 *>(buf + lane * kStagePitch);
     tc_fence_after();
 #pragma unroll
@@ -394,7 +398,7 @@ __device__ __forceinline__ void cluster_merge_exchange(const DecodeParams &p, Co
 #pragma unroll
             for (int j = 0; j < 32; ++j) ov[j] = 0u;
         }
-        const uint4 *r4 = reinterpret_cast<const uint4 *>(theirs + c2 * 128);
+        const uint4 *r4 = reinterpret_cast<const uint4 *>(theirs + c2 * kChunkBytes);
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const uint4 ra = r4[2 * j], rb = r4[2 * j + 1];
@@ -1087,9 +1091,11 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(grp ? p_full_leader1 : p_full_leader0);
         }
+        // The row sums are final as soon as the last tile's weights are written, before its P V has
+        // run: their exchange and what follows from them overlap that last P V.
         if (ok) {
-            // the last tile's P V has retired and its reference is the final one
-            ok = mbar_wait(&ctl->pv_done[(tiles - 1) & 1], ((tiles - 1) >> 1) & 1) && mbar_wait(&ctl->ref_bar, (tiles - 1) & 1);
+            // the reference after the last tile is the final one
+            ok = mbar_wait(&ctl->ref_bar, (tiles - 1) & 1);
             ok = __all_sync(0xffffffffu, ok);
         }
         if (ok) {
@@ -1099,28 +1105,39 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
                 m_ref = ref_final;
             }
         }
-        constexpr int xs = 0;                                  // exchange slot of the final row sums
+        // Slot of a group's partial row sums: the group's row-maximum slots of the parity it did NOT
+        // use for its last tile.  Every thread of the group has passed the exchange barrier of that
+        // last tile, which each thread reached only after reading the slots of the tile before, so
+        // nobody reads them any more (a group without tiles never used its slots at all).
+        auto sum_slot = [&](int g) -> float * {
+            const int last = (tiles - 1) - ((((tiles - 1) & 1) != g) ? 1 : 0);      // the group's last tile, -1 if none
+            const int parity = last >= 0 ? (((last >> 1) & 1) ^ 1) : 0;
+            return &ctl->xchg[0][0][0] + ((g * 2 + parity) * 2) * 64;                // [half][row]
+        };
+        float lt = 0.f;
         if (ok) {
-            // total row sum: add the partial sums of the row's other three threads (the groups'
-            // exchange slots are dead by now: the last P V could only be issued after every warp of
-            // its group had read its partner's maximum and written its weights)
-            ctl->xchg[xs][part][row] = l;
+            sum_slot(grp)[half * 64 + row] = l;
             mbar_arrive(&ctl->x_bar);
             ok = mbar_wait(&ctl->x_bar, 0);
             ok = __all_sync(0xffffffffu, ok);
         }
-        if (ok && p.cluster_merge) {
-            // every MMA of the pair has retired and every copy has landed: the partner in the other
-            // split may overwrite this CTA's operand tiles from now on
-            if (warp == 2 && lane == 0) mbar_arrive_cluster(map_to_rank(smem_u32(&ctl->ready_bar), crank ^ 2u));
-            // the result stays in tensor memory: the exchange after the main loop normalises it and
-            // hands half of it to the CTA that serves the same heads in the other split
-            const float lt = (ctl->xchg[xs][0][row] + ctl->xchg[xs][1][row]) + (ctl->xchg[xs][2][row] + ctl->xchg[xs][3][row]);
+        if (ok) {
+            const float *s0 = sum_slot(0), *s1 = sum_slot(1);
+            lt = (s0[row] + s0[64 + row]) + (s1[row] + s1[64 + row]);
             cm_inv = lt > 0.f ? 1.f / lt : 0.f;
             cm_lse = lt > 0.f ? (m_ref + log2f(lt)) * kLn2 : -INFINITY;
+            // now the last tile's P V
+            ok = mbar_wait(&ctl->pv_done[(tiles - 1) & 1], ((tiles - 1) >> 1) & 1);
+            ok = __all_sync(0xffffffffu, ok);
+        }
+        if (ok && p.cluster_merge) {
+            // every MMA of the pair has retired and every copy has landed: the partner in the other
+            // split may overwrite this CTA's operand tiles from now on.  The result stays in tensor
+            // memory: the exchange after the main loop normalises it and hands half of it to the CTA
+            // that serves the same heads in the other split.
+            if (warp == 2 && lane == 0) mbar_arrive_cluster(map_to_rank(smem_u32(&ctl->ready_bar), crank ^ 2u));
         } else if (ok) {
             tc_fence_after();
-            const float lt = (ctl->xchg[xs][0][row] + ctl->xchg[xs][1][row]) + (ctl->xchg[xs][2][row] + ctl->xchg[xs][3][row]);
             c2_store_result(p, smem, tmem, warp, lane, b, s, h0, head_rows, lt, m_ref);
             const bool final_out = p.splits == 1;
             // with the in-kernel merge the partial results must be visible before this CTA is counted
