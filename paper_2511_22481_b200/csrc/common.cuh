@@ -81,7 +81,24 @@ struct Selection {
     int vstart;            // ranges only: entry of position rs
     int sink_pages, ring_pages;   // ranges over a rolling cache (ring_pages > 0)
     bool bad;              // the length breaks the contract (n was set to 0)
+    uint64_t keep;         // L2 policy of the index loads (see ldg_index)
 };
+
+// Index data (token positions, page ids) is a few bytes per token and is read by several warps of
+// both CTAs that serve a request; the cache rows stream through L2 at a thousand times the volume
+// and would push it out between two uses.  Its loads therefore ask L2 to evict these lines last.
+__device__ __forceinline__ uint64_t index_load_policy()
+{
+    uint64_t policy;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(policy));
+    return policy;
+}
+__device__ __forceinline__ int32_t ldg_index(const int32_t *ptr, uint64_t policy)
+{
+    int32_t v;
+    asm volatile("ld.global.nc.L2::cache_hint.b32 %0, [%1], %2;" : "=r"(v) : "l"(ptr), "l"(policy));
+    return v;
+}
 
 __device__ __forceinline__ Selection load_selection(const DecodeParams &p, int b)
 {
@@ -90,6 +107,7 @@ __device__ __forceinline__ Selection load_selection(const DecodeParams &p, int b
     s.ns = s.rs = s.vstart = 0;
     s.sink_pages = p.sink_pages;
     s.ring_pages = p.ring_pages;
+    s.keep = index_load_policy();
     if (p.sel_idx != nullptr) {
         s.list = p.sel_idx + (size_t)b * p.max_sel;
         s.n = __ldg(p.sel_len + b);
@@ -125,7 +143,7 @@ __device__ __forceinline__ bool is_padding(const Selection &s, int32_t t)
 
 __device__ __forceinline__ int32_t selection_at(const Selection &s, int j)
 {
-    if (s.list != nullptr) return __ldg(s.list + j);
+    if (s.list != nullptr) return ldg_index(s.list + j, s.keep);
     if (j >= s.ns && j < s.vstart) return kSelectionPad;
     const int32_t t = j < s.ns ? j : s.rs + (j - s.vstart);
     return s.ring_pages > 0 ? rolling_position(t, s.sink_pages, s.ring_pages) : t;

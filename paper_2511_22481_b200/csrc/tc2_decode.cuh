@@ -658,8 +658,8 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
         x.t1 = (tile < tiles && j1 < end) ? selection_at(selection, j1) : -1;
     };
     auto stage_pages = [&](TileIdx &x) {
-        x.pg0 = (x.t0 >= 0 && x.t0 / kPage < p.max_pages) ? __ldg(pt + x.t0 / kPage) : -1;
-        x.pg1 = (x.t1 >= 0 && x.t1 / kPage < p.max_pages) ? __ldg(pt + x.t1 / kPage) : -1;
+        x.pg0 = (x.t0 >= 0 && x.t0 / kPage < p.max_pages) ? ldg_index(pt + x.t0 / kPage, selection.keep) : -1;
+        x.pg1 = (x.t1 >= 0 && x.t1 / kPage < p.max_pages) ? ldg_index(pt + x.t1 / kPage, selection.keep) : -1;
     };
     // row_lo / row_hi: pool rows of tokens lane and lane+32 (a masked token repeats the row of the
     // tile's first valid token: real cache contents, multiplied by a weight of exactly zero);
@@ -836,12 +836,14 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
                 if (t < tiles && j0 + kC2Tile <= end) {
                     const int first = selection_at(selection, j0), last = selection_at(selection, j0 + kC2Tile - 1);
                     if (first >= 0 && first % kPage == 0 && last == first + kC2Tile - 1 && first / kPage < p.max_pages) {
-                        const int pg = __ldg(pt + first / kPage);
+                        const int pg = ldg_index(pt + first / kPage, selection.keep);
                         if (pg >= 0 && (int64_t)pg < p.num_pages) row = pg * kPage;
                     }
                 }
                 const int count = min(32, tiles - t0);
                 bool ok = true;
+                // nothing to pace out where no tile of the batch is a whole page (token-level selections)
+                if (!__any_sync(0xffffffffu, row >= 0)) continue;
                 for (int k = 0; ok && k < count; ++k) {
                     // tile i is prefetched once the K loads of tile i - kPrefetchAhead have started (a
                     // monotonic counter, polled with a bounded number of naps)
@@ -969,7 +971,6 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
         const int sub = warp >= 8 ? 1 : 0;
         const int row = (quarter & 1) * 32 + lane;          // head row within this CTA
         const int half = quarter >> 1;                      // token half of S / column half of O
-        const int part = half * 2 + sub;                    // which quarter of the tile's tokens
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
         const uint32_t s_empty_leader = map_to_rank(smem_u32(&ctl->s_empty[0]), leader);   // [1], [2] follow at +8, +16
         const uint32_t p_full_leader0 = map_to_rank(smem_u32(&ctl->p_full[0]), leader);

@@ -274,8 +274,8 @@ tc2q8_decode_kernel(const __grid_constant__ CUtensorMap q_nope_map, const __grid
         x.t1 = (tile < tiles && j1 < end) ? selection_at(selection, j1) : -1;
     };
     auto stage_pages = [&](TileIdx &x) {
-        x.pg0 = (x.t0 >= 0 && x.t0 / kPage < p.max_pages) ? __ldg(pt + x.t0 / kPage) : -1;
-        x.pg1 = (x.t1 >= 0 && x.t1 / kPage < p.max_pages) ? __ldg(pt + x.t1 / kPage) : -1;
+        x.pg0 = (x.t0 >= 0 && x.t0 / kPage < p.max_pages) ? ldg_index(pt + x.t0 / kPage, selection.keep) : -1;
+        x.pg1 = (x.t1 >= 0 && x.t1 / kPage < p.max_pages) ? ldg_index(pt + x.t1 / kPage, selection.keep) : -1;
     };
     auto stage_rows = [&](int tile, const TileIdx &x, int &row_lo, int &row_hi, uint64_t &mask, bool &contig,
                           bool &contig_lo, bool &contig_hi, bool &any_bad) {
@@ -444,12 +444,13 @@ tc2q8_decode_kernel(const __grid_constant__ CUtensorMap q_nope_map, const __grid
                 if (t < tiles && j0 + kC2Tile <= end) {
                     const int first = selection_at(selection, j0), last = selection_at(selection, j0 + kC2Tile - 1);
                     if (first >= 0 && first % kPage == 0 && last == first + kC2Tile - 1 && first / kPage < p.max_pages) {
-                        const int pg = __ldg(pt + first / kPage);
+                        const int pg = ldg_index(pt + first / kPage, selection.keep);
                         if (pg >= 0 && (int64_t)pg < p.num_pages) row = pg * kPage;
                     }
                 }
                 const int count = min(32, tiles - t0);
                 bool ok = true;
+                if (!__any_sync(0xffffffffu, row >= 0)) continue;
                 for (int k = 0; ok && k < count; ++k) {
                     const int i = t0 + k;
                     const volatile int32_t *progress = &ctl->k_progress;
