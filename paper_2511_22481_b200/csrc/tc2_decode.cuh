@@ -131,9 +131,13 @@ __device__ __forceinline__ void cluster_sync_relaxed()
     asm volatile("barrier.cluster.arrive.relaxed.aligned;\n\tbarrier.cluster.wait.aligned;" ::: "memory");
 }
 
-__device__ __forceinline__ void cluster_sync_all()
+// Rendezvous of the cluster after the barriers were initialised.  The initialising thread has
+// issued the barrier-init fence, so the arrive needs no release of its own (a release-ordered
+// arrive cost half a microsecond of every launch); nothing else that the other CTAs read was
+// written before it.
+__device__ __forceinline__ void cluster_sync_after_init()
 {
-    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.arrive.relaxed.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
 // 3-D box {64 columns, box rows, n column panels} loaded by one CTA of a pair: lands panel-major,
@@ -617,7 +621,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
     }
     tc_fence_before();
     __syncthreads();
-    cluster_sync_all();
+    cluster_sync_after_init();
     tc_fence_after();
     // Programmatic dependent launch, both ways.  This grid may have been scheduled while the
     // kernel before it in the stream was still finishing: nothing in global memory is touched

@@ -242,7 +242,7 @@ tc2q8_decode_kernel(const __grid_constant__ CUtensorMap q_nope_map, const __grid
     }
     tc_fence_before();
     __syncthreads();
-    cluster_sync_all();
+    cluster_sync_after_init();
     tc_fence_after();
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
