@@ -431,12 +431,16 @@ def main():
     sampler.start()                           # before the warm-up, so that short timed regions are sampled too
     for i in range(args.warmup):
         step(i)
-    barrier()
+    # what the harness itself needs is made before the timed region opens: the events exist (a first
+    # record creates them) and the list of per-step calls is built
     t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_begin.record()
+    t_end.record()
+    calls = [planned[(args.warmup + i) % clones] for i in range(args.steps)] if planned is not None else None
+    barrier()
     t_begin.record()
     host_t0 = time.perf_counter()
     if planned is not None:
-        calls = [planned[(args.warmup + i) % clones] for i in range(args.steps)]
         for call in calls:
             call()
     else:
