@@ -331,6 +331,8 @@ def main():
                     help="tc: tensor-core kernel (the product path); simt: plain-FMA bring-up kernel")
     ap.add_argument("--clones", type=int, default=6, help="KV pool copies rotated to keep L2 cold")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--e2e-lanes", type=int, default=2,
+                    help="end-to-end leg: how many steps are in flight, each on its own stream and buffers")
     ap.add_argument("--workload", default="config2", help=WORKLOAD_HELP)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
@@ -489,18 +491,48 @@ def main():
             out_h.copy_(plan.out, non_blocking=True)
             lse_h.copy_(plan.lse, non_blocking=True)
     else:
+        # Two steps in flight: consecutive steps go to two streams in turn, each with its own staging
+        # area, host result buffers and workspace, so that the copies out of one step overlap the
+        # copies in of the next (PCIe carries both directions at once).  Every step still moves all of
+        # its inputs in and all of its results out.
+        lanes = []
+        for k in range(max(1, args.e2e_lanes)):
+            lanes.append({
+                "stream": torch.cuda.Stream(device=dev),
+                "staging": staging if k == 0 else torch.empty_like(staging),
+                "out_h": out_h if k == 0 else torch.empty_like(out_h).pin_memory(),
+                "lse_h": lse_h if k == 0 else torch.empty_like(lse_h).pin_memory(),
+                "ws": plan.workspace if k == 0 or plan.workspace is None else torch.empty_like(plan.workspace),
+            })
+        e2e_lanes = len(lanes)
+
         def e2e_step(i):
-            B.omni_sparse_mla_decode_host(plan.desc, q_h, pools[i % clones], pt_h, si_h, sl_h, out_h,
-                                          lse_h, staging, plan.workspace, plan.status)
+            ln = lanes[i % e2e_lanes]
+            B.omni_sparse_mla_decode_host(plan.desc, q_h, pools[i % clones], pt_h, si_h, sl_h, ln["out_h"],
+                                          ln["lse_h"], ln["staging"], ln["ws"], plan.status, ln["stream"])
+
+    def fork_lanes():
+        if not q8:
+            for ln in lanes:
+                ln["stream"].wait_stream(torch.cuda.current_stream())
+
+    def join_lanes():
+        if not q8:
+            for ln in lanes:
+                torch.cuda.current_stream().wait_stream(ln["stream"])
 
     e2e_steps = args.steps
+    fork_lanes()
     for i in range(args.warmup):
         e2e_step(i)
+    join_lanes()
     barrier()
     e_begin, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e_begin.record()
+    fork_lanes()
     for i in range(e2e_steps):
         e2e_step(args.warmup + i)
+    join_lanes()
     e_end.record()
     barrier()
     e2e_ms_total = e_begin.elapsed_time(e_end)
@@ -546,7 +578,10 @@ def main():
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "note": "omni_sparse_mla_decode_host: q, page_table, sel_idx, sel_len copied from pinned "
                             "host memory and out, lse copied back every step; the KV cache is persistent "
-                            "device state"},
+                            "device state" + ("" if q8 else "; consecutive steps take turns on several "
+                                                      "streams (own staging, result buffers and workspace each), so one "
+                                                      "step's copies out overlap the next step's copies in"),
+                    "steps_in_flight": 1 if q8 else max(1, args.e2e_lanes)},
             "gpu_launches": launches_per_step * args.steps,
             "host_us_per_call": round(host_us_per_call, 3),
             "launch_bound": bool(host_us_per_call > 0.9 * ms_per_step * 1e3),

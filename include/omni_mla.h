@@ -14,8 +14,8 @@
  *     The library allocates no device memory and keeps no per-call state.  What it does keep,
  *     per process: per-device facts looked up once (SM count, kernel attributes, how many
  *     merging clusters fit), a table of tensor-map encodings keyed by (base address, sizes)
- *     so that repeated calls on the same buffers skip the encoding, one side stream per
- *     device for omni_sparse_mla_decode_host, the address of the static scratch array of
+ *     so that repeated calls on the same buffers skip the encoding, up to four side streams per
+ *     device for omni_sparse_mla_decode_host (chosen by the caller's stream), the address of the static scratch array of
  *     omni_sparse_mla_decode_static, and the two event handles of
  *     omni_sparse_mla_set_profile_events.  All of it is guarded for use from several host
  *     threads except the profile events.

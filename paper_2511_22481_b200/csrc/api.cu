@@ -671,16 +671,21 @@ static size_t host_half_workspace(const omni_mla_desc_t *desc, int half)
     return align_up(workspace_need(&d, choose_splits(&d, device_info().sm_count)), 256);
 }
 
-static cudaStream_t host_side_stream()
+// Side streams of the host-buffer entry point: a few per device, chosen by the caller's stream, so
+// that calls in flight on different streams do not queue their second halves behind one another.
+constexpr int kHostSideStreams = 4;
+static cudaStream_t host_side_stream(cudaStream_t caller)
 {
     static std::mutex lock;
-    static cudaStream_t streams[64] = {};
+    static cudaStream_t streams[64][kHostSideStreams] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    const uintptr_t h = reinterpret_cast<uintptr_t>(caller);
+    const int slot = (int)(((h >> 4) ^ (h >> 12) ^ (h >> 20)) % kHostSideStreams);
     std::lock_guard<std::mutex> guard(lock);
-    if (!streams[dev] && cudaStreamCreateWithFlags(&streams[dev], cudaStreamNonBlocking) != cudaSuccess)
-        streams[dev] = nullptr;
-    return streams[dev];
+    if (!streams[dev][slot] && cudaStreamCreateWithFlags(&streams[dev][slot], cudaStreamNonBlocking) != cudaSuccess)
+        streams[dev][slot] = nullptr;
+    return streams[dev][slot];
 }
 
 size_t omni_sparse_mla_host_staging_bytes(const omni_mla_desc_t *desc)
@@ -743,7 +748,7 @@ omni_status_t omni_sparse_mla_decode_host(const omni_mla_desc_t *desc, const voi
         return OMNI_OK;
     };
 
-    cudaStream_t side = host_pipelined(desc) ? host_side_stream() : nullptr;
+    cudaStream_t side = host_pipelined(desc) ? host_side_stream(stream) : nullptr;
     if (!side) {
         if (!copy_q(0, B, stream) || !copy_indices(stream)) return OMNI_ERR_CUDA;
         return decode_and_copy_out(*desc, 0, workspace, workspace_bytes, stream);
