@@ -331,6 +331,36 @@ def test_host_buffer_entry_point_two_halves(flags, batch):
     compare(out_h, lse_h, ref_out, ref_lse, "host entry point, two halves")
 
 
+def test_host_buffer_entry_point_two_calls_in_flight(flags):
+    """Two calls on two streams at once, each with its own staging area, result buffers and
+    workspace (how the benchmark's end-to-end leg keeps two steps in flight): each result is the
+    oracle's, whichever side streams the library picked for them."""
+    ws_list = [W.config4_topk(DEV, batch=8, ctx_pages=32, k=300), W.config4_topk(DEV, batch=9, ctx_pages=32, k=280)]
+    pin = lambda t: t.cpu().pin_memory()
+    lanes = []
+    for w in ws_list:
+        desc = B.make_desc(w.batch, w.heads, w.num_pages, w.max_pages_per_req, w.max_sel, w.scale, flags=flags)
+        lanes.append(dict(
+            w=w, desc=desc, stream=torch.cuda.Stream(device=DEV),
+            staging=torch.empty(B.omni_sparse_mla_host_staging_bytes(desc), dtype=torch.uint8, device=DEV),
+            ws=torch.empty(max(1, B.omni_sparse_mla_workspace_bytes(desc)), dtype=torch.uint8, device=DEV),
+            host=[pin(t) for t in (w.q, w.page_table, w.sel_idx, w.sel_len)],
+            out_h=torch.full((w.batch, w.heads, 512), float("nan"), dtype=torch.bfloat16).pin_memory(),
+            lse_h=torch.full((w.batch, w.heads), float("nan"), dtype=torch.float32).pin_memory(),
+            status=torch.zeros(1, dtype=torch.int32, device=DEV)))
+    torch.cuda.synchronize()
+    for _ in range(3):
+        for ln in lanes:
+            q, pt, si, sl = ln["host"]
+            B.omni_sparse_mla_decode_host(ln["desc"], q, ln["w"].kv_cache, pt, si, sl, ln["out_h"], ln["lse_h"],
+                                          ln["staging"], ln["ws"], ln["status"], ln["stream"])
+    for ln in lanes:
+        ln["stream"].synchronize()                       # each caller's stream alone covers its call
+        assert int(ln["status"].item()) == 0
+        ref_out, ref_lse, _ = oracle_subset(ln["w"])
+        compare(ln["out_h"], ln["lse_h"], ref_out, ref_lse, "host entry point, two calls in flight")
+
+
 # ------------------------------------------------------------------ full benchmark sizes
 
 def test_config2_full_size_every_row(flags):
