@@ -588,7 +588,7 @@ def main():
             "roofline": {"bound": "hbm", "achieved": round(achieved, 2), "peak": peaks["hbm"],
                          "unit": "GB/s", "frac": round(achieved / peaks["hbm"], 4),
                          "traffic": _recorded_traffic(khash), "peak_source": peaks["source"],
-                         "kernel": "sparse_mla_decode main kernel (tc2_decode_kernel for 128 heads)", "kernel_us_mean": round(kmean * 1e3, 3),
+                         "kernel": "sparse_mla_decode main kernel (128 heads: tc2_decode_cm_kernel where two splits merge inside a cluster, as on the bench workload, else tc2_decode_kernel)", "kernel_us_mean": round(kmean * 1e3, 3),
                          "kernel_us_bracketed_min": round(min(kern_ms) * 1e3, 3),
                          "kernel_us_bracketed_mean": round(kbracket * 1e3, 3),
                          "kernel_us_source": ("timed region / steps (one launch per step)" if launches_per_step == 1

@@ -556,10 +556,13 @@ __device__ __forceinline__ void c2_store_result(const DecodeParams &p, uint8_t *
     }
 }
 
-__global__ void __launch_bounds__(kC2Threads, 1)
-tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
-                  const __grid_constant__ CUtensorMap kv_k_map, const __grid_constant__ CUtensorMap kv_v_map,
-                  const __grid_constant__ CUtensorMap kv_tile_map, DecodeParams p)
+// The kernel body in two instances: kClusterMerge = true, the two splits of a request merged
+// inside a cluster of two pairs; false, every other form (no split, merge kernel, fused merge).
+// Each instance carries only its own merge and epilogue code.
+template <bool kClusterMerge>
+__device__ __forceinline__ void tc2_decode_body(const CUtensorMap &q_map, const CUtensorMap &kv_k_map,
+                                                const CUtensorMap &kv_v_map, const CUtensorMap &kv_tile_map,
+                                                const DecodeParams &p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = smem_raw;
@@ -578,8 +581,8 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
     const uint16_t pair_mask = (uint16_t)(3u << leader);
 
     const int pair = blockIdx.x >> 1;
-    const int s = p.cluster_merge ? (int)(crank >> 1) : pair % p.splits;
-    int b = p.cluster_merge ? (int)(blockIdx.x >> 2) : pair / p.splits;
+    const int s = kClusterMerge ? (int)(crank >> 1) : pair % p.splits;
+    int b = kClusterMerge ? (int)(blockIdx.x >> 2) : pair / p.splits;
     const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;  // warp-uniform
     const int h0 = (int)rank * kTcHeads;
     const int head_rows = min(kTcHeads, p.heads - h0);
@@ -629,7 +632,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
     // may be scheduled as soon as resources allow; it waits in the same way before it reads.
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (p.longest_first) b = c2_request_by_length_rank(p, reinterpret_cast<int *>(smem), &ctl->merge_flag, b);
+    if (!kClusterMerge && p.longest_first) b = c2_request_by_length_rank(p, reinterpret_cast<int *>(smem), &ctl->merge_flag, b);
     const Selection selection = load_selection(p, b);
     const int n = selection.n;
     const bool bad_len = selection.bad;
@@ -639,7 +642,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
 
     const bool active = tiles > 0;
     if (!active && bad_len && threadIdx.x == 0 && crank == 0) flag_status(p.status, OMNI_DEV_BAD_INDEX);
-    if (!active && !p.cluster_merge) {
+    if (!kClusterMerge && !active) {
         // empty split (the same decision in both CTAs of the pair): zeros and -inf, no pipeline
         c2_store_empty(p, b, s, h0, head_rows, warp, lane);
     }
@@ -1135,13 +1138,13 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
             ok = mbar_wait(&ctl->pv_done[(tiles - 1) & 1], ((tiles - 1) >> 1) & 1);
             ok = __all_sync(0xffffffffu, ok);
         }
-        if (ok && p.cluster_merge) {
+        if (kClusterMerge && ok) {
             // every MMA of the pair has retired and every copy has landed: the partner in the other
             // split may overwrite this CTA's operand tiles from now on.  The result stays in tensor
             // memory: the exchange after the main loop normalises it and hands half of it to the CTA
             // that serves the same heads in the other split.
             if (warp == 2 && lane == 0) mbar_arrive_cluster(map_to_rank(smem_u32(&ctl->ready_bar), crank ^ 2u));
-        } else if (ok) {
+        } else if (!kClusterMerge && ok) {
             tc_fence_after();
             c2_store_result(p, smem, tmem, warp, lane, b, s, h0, head_rows, lt, m_ref);
             const bool final_out = p.splits == 1;
@@ -1160,7 +1163,7 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
         // a wait ran out: give copies that are still in flight time to land before anyone exits
         for (int i = 0; i < 200; ++i) __nanosleep(1000);
     }
-    if (p.cluster_merge) cluster_merge_exchange(p, ctl, smem, tmem, b, s, crank, h0, head_rows, active, softmax_ok, cm_lse, cm_inv);
+    if (kClusterMerge) cluster_merge_exchange(p, ctl, smem, tmem, b, s, crank, h0, head_rows, active, softmax_ok, cm_lse, cm_inv);
     tc_fence_before();
     __syncthreads();
     // Tensor memory was allocated for the pair, so it is released only when both CTAs are done
@@ -1179,10 +1182,26 @@ tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
     }
     // the bulk copy a CTA sent to its partner reads this CTA's shared memory: nobody leaves
     // before every CTA of the cluster has received its block
-    if (p.cluster_merge) cluster_sync_relaxed();
+    if (kClusterMerge) cluster_sync_relaxed();
     // ---- split merge by whichever CTA finishes a (request, head half) last ---------------
-    if (p.splits > 1 && p.counters != nullptr)
+    if (!kClusterMerge && p.splits > 1 && p.counters != nullptr)
         merge_if_last(p, b, (int)rank, 2, h0, head_rows, reinterpret_cast<float *>(smem), &ctl->merge_flag);
+}
+
+__global__ void __launch_bounds__(kC2Threads, 1)
+tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
+                  const __grid_constant__ CUtensorMap kv_k_map, const __grid_constant__ CUtensorMap kv_v_map,
+                  const __grid_constant__ CUtensorMap kv_tile_map, DecodeParams p)
+{
+    tc2_decode_body<false>(q_map, kv_k_map, kv_v_map, kv_tile_map, p);
+}
+
+__global__ void __launch_bounds__(kC2Threads, 1)
+tc2_decode_cm_kernel(const __grid_constant__ CUtensorMap q_map,
+                     const __grid_constant__ CUtensorMap kv_k_map, const __grid_constant__ CUtensorMap kv_v_map,
+                     const __grid_constant__ CUtensorMap kv_tile_map, DecodeParams p)
+{
+    tc2_decode_body<true>(q_map, kv_k_map, kv_v_map, kv_tile_map, p);
 }
 
 // Clusters of two pairs (cluster merge) that can be resident at once on the current device, or 0.
@@ -1196,7 +1215,7 @@ inline int tc2_max_merge_clusters()
     std::lock_guard<std::mutex> lock(mu);
     if (!known[dev]) {
         int n = 0;
-        if (cudaFuncSetAttribute(tc2_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kC2SmemBytes) == cudaSuccess) {
+        if (cudaFuncSetAttribute(tc2_decode_cm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kC2SmemBytes) == cudaSuccess) {
             cudaLaunchConfig_t cfg = {};
             cfg.gridDim = dim3(4 * 64);
             cfg.blockDim = dim3(kC2Threads);
@@ -1208,7 +1227,7 @@ inline int tc2_max_merge_clusters()
             attr[0].val.clusterDim.z = 1;
             cfg.attrs = attr;
             cfg.numAttrs = 1;
-            if (cudaOccupancyMaxActiveClusters(&n, tc2_decode_kernel, &cfg) != cudaSuccess) {
+            if (cudaOccupancyMaxActiveClusters(&n, tc2_decode_cm_kernel, &cfg) != cudaSuccess) {
                 cudaGetLastError();
                 n = 0;
             }
@@ -1228,7 +1247,9 @@ inline bool tc2_prepare_device()
     std::lock_guard<std::mutex> lock(mu);
     if (!attr_set[dev]) {
         if (cudaFuncSetAttribute(tc2_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kC2SmemBytes) !=
-            cudaSuccess)
+                cudaSuccess ||
+            cudaFuncSetAttribute(tc2_decode_cm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kC2SmemBytes) !=
+                cudaSuccess)
             return false;
         attr_set[dev] = true;
     }
@@ -1264,9 +1285,10 @@ inline omni_status_t tc2_launch(const CUtensorMap *maps, const DecodeParams &p, 
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, tc2_decode_kernel, maps[0], maps[1], maps[2], maps[3], p) == cudaSuccess
-               ? OMNI_OK
-               : OMNI_ERR_CUDA;
+    const cudaError_t err = p.cluster_merge
+                                ? cudaLaunchKernelEx(&cfg, tc2_decode_cm_kernel, maps[0], maps[1], maps[2], maps[3], p)
+                                : cudaLaunchKernelEx(&cfg, tc2_decode_kernel, maps[0], maps[1], maps[2], maps[3], p);
+    return err == cudaSuccess ? OMNI_OK : OMNI_ERR_CUDA;
 }
 
 }  // namespace omni
