@@ -558,8 +558,9 @@ __device__ __forceinline__ void c2_store_result(const DecodeParams &p, uint8_t *
 
 // The kernel body in two instances: kClusterMerge = true, the two splits of a request merged
 // inside a cluster of two pairs; false, every other form (no split, merge kernel, fused merge).
-// Each instance carries only its own merge and epilogue code.
-template <bool kClusterMerge>
+// kRanges = false: the selection is the caller's index list; true: Eq. 2's two ranges (with or
+// without a rolling cache).  Each instance carries only its own merge, epilogue and index code.
+template <bool kClusterMerge, bool kRanges>
 __device__ __forceinline__ void tc2_decode_body(const CUtensorMap &q_map, const CUtensorMap &kv_k_map,
                                                 const CUtensorMap &kv_v_map, const CUtensorMap &kv_tile_map,
                                                 const DecodeParams &p)
@@ -634,6 +635,7 @@ __device__ __forceinline__ void tc2_decode_body(const CUtensorMap &q_map, const 
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (!kClusterMerge && p.longest_first) b = c2_request_by_length_rank(p, reinterpret_cast<int *>(smem), &ctl->merge_flag, b);
     const Selection selection = load_selection(p, b);
+    __builtin_assume(kRanges ? selection.list == nullptr : selection.list != nullptr);
     const int n = selection.n;
     const bool bad_len = selection.bad;
     int begin, end;
@@ -1188,20 +1190,24 @@ __device__ __forceinline__ void tc2_decode_body(const CUtensorMap &q_map, const 
         merge_if_last(p, b, (int)rank, 2, h0, head_rows, reinterpret_cast<float *>(smem), &ctl->merge_flag);
 }
 
-__global__ void __launch_bounds__(kC2Threads, 1)
-tc2_decode_kernel(const __grid_constant__ CUtensorMap q_map,
-                  const __grid_constant__ CUtensorMap kv_k_map, const __grid_constant__ CUtensorMap kv_v_map,
-                  const __grid_constant__ CUtensorMap kv_tile_map, DecodeParams p)
-{
-    tc2_decode_body<false>(q_map, kv_k_map, kv_v_map, kv_tile_map, p);
-}
+#define OMNI_C2_KERNEL(name, cluster_merge, ranges)                                                                    \
+    __global__ void __launch_bounds__(kC2Threads, 1)                                                                   \
+    name(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap kv_k_map,                      \
+         const __grid_constant__ CUtensorMap kv_v_map, const __grid_constant__ CUtensorMap kv_tile_map, DecodeParams p) \
+    {                                                                                                                  \
+        tc2_decode_body<cluster_merge, ranges>(q_map, kv_k_map, kv_v_map, kv_tile_map, p);                             \
+    }
+OMNI_C2_KERNEL(tc2_decode_kernel, false, false)
+OMNI_C2_KERNEL(tc2_decode_cm_kernel, true, false)
+OMNI_C2_KERNEL(tc2_decode_rng_kernel, false, true)
+OMNI_C2_KERNEL(tc2_decode_cm_rng_kernel, true, true)
+#undef OMNI_C2_KERNEL
 
-__global__ void __launch_bounds__(kC2Threads, 1)
-tc2_decode_cm_kernel(const __grid_constant__ CUtensorMap q_map,
-                     const __grid_constant__ CUtensorMap kv_k_map, const __grid_constant__ CUtensorMap kv_v_map,
-                     const __grid_constant__ CUtensorMap kv_tile_map, DecodeParams p)
+using C2KernelFn = void (*)(CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, DecodeParams);
+inline C2KernelFn tc2_kernel_for(bool cluster_merge, bool ranges)
 {
-    tc2_decode_body<true>(q_map, kv_k_map, kv_v_map, kv_tile_map, p);
+    return cluster_merge ? (ranges ? tc2_decode_cm_rng_kernel : tc2_decode_cm_kernel)
+                         : (ranges ? tc2_decode_rng_kernel : tc2_decode_kernel);
 }
 
 // Clusters of two pairs (cluster merge) that can be resident at once on the current device, or 0.
@@ -1246,11 +1252,10 @@ inline bool tc2_prepare_device()
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
     std::lock_guard<std::mutex> lock(mu);
     if (!attr_set[dev]) {
-        if (cudaFuncSetAttribute(tc2_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kC2SmemBytes) !=
-                cudaSuccess ||
-            cudaFuncSetAttribute(tc2_decode_cm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kC2SmemBytes) !=
-                cudaSuccess)
-            return false;
+        for (int k = 0; k < 4; ++k)
+            if (cudaFuncSetAttribute(tc2_kernel_for((k & 1) != 0, (k & 2) != 0), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     kC2SmemBytes) != cudaSuccess)
+                return false;
         attr_set[dev] = true;
     }
     return true;
@@ -1285,9 +1290,8 @@ inline omni_status_t tc2_launch(const CUtensorMap *maps, const DecodeParams &p, 
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    const cudaError_t err = p.cluster_merge
-                                ? cudaLaunchKernelEx(&cfg, tc2_decode_cm_kernel, maps[0], maps[1], maps[2], maps[3], p)
-                                : cudaLaunchKernelEx(&cfg, tc2_decode_kernel, maps[0], maps[1], maps[2], maps[3], p);
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, tc2_kernel_for(p.cluster_merge != 0, p.sel_idx == nullptr), maps[0], maps[1],
+                                               maps[2], maps[3], p);
     return err == cudaSuccess ? OMNI_OK : OMNI_ERR_CUDA;
 }
 
