@@ -178,10 +178,12 @@ __device__ __noinline__ void gather_v_rows_q8(uint32_t dst, const char *kv_cols,
     cp_async_commit();
 }
 
-__global__ void __launch_bounds__(kC2Threads, 1)
-tc2q8_decode_kernel(const __grid_constant__ CUtensorMap q_nope_map, const __grid_constant__ CUtensorMap q_rope_map,
-                    const __grid_constant__ CUtensorMap kv_k_map, const __grid_constant__ CUtensorMap kv_v_map,
-                    const __grid_constant__ CUtensorMap kv_page_map, DecodeParams p)
+// Two instances, as for the bf16 kernel: with and without the in-cluster merge of two splits, each
+// carrying only its own merge and epilogue code.  The 8-bit entry point takes an index list only.
+template <bool kClusterMerge>
+__device__ __forceinline__ void tc2q8_decode_body(const CUtensorMap &q_nope_map, const CUtensorMap &q_rope_map,
+                                                  const CUtensorMap &kv_k_map, const CUtensorMap &kv_v_map,
+                                                  const CUtensorMap &kv_page_map, const DecodeParams &p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = smem_raw;
@@ -198,8 +200,8 @@ tc2q8_decode_kernel(const __grid_constant__ CUtensorMap q_nope_map, const __grid
     const uint16_t pair_mask = (uint16_t)(3u << leader);
 
     const int pair = blockIdx.x >> 1;
-    const int s = p.cluster_merge ? (int)(crank >> 1) : pair % p.splits;
-    int b = p.cluster_merge ? (int)(blockIdx.x >> 2) : pair / p.splits;
+    const int s = kClusterMerge ? (int)(crank >> 1) : pair % p.splits;
+    int b = kClusterMerge ? (int)(blockIdx.x >> 2) : pair / p.splits;
     const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;  // warp-uniform
     const int h0 = (int)rank * kTcHeads;
     const int head_rows = min(kTcHeads, p.heads - h0);
@@ -246,8 +248,9 @@ tc2q8_decode_kernel(const __grid_constant__ CUtensorMap q_nope_map, const __grid
     tc_fence_after();
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (p.longest_first) b = c2_request_by_length_rank(p, reinterpret_cast<int *>(smem), &ctl->merge_flag, b);
+    if (!kClusterMerge && p.longest_first) b = c2_request_by_length_rank(p, reinterpret_cast<int *>(smem), &ctl->merge_flag, b);
     const Selection selection = load_selection(p, b);
+    __builtin_assume(selection.list != nullptr);
     const int n = selection.n;
     const bool bad_len = selection.bad;
     int begin, end;
@@ -256,7 +259,7 @@ tc2q8_decode_kernel(const __grid_constant__ CUtensorMap q_nope_map, const __grid
 
     const bool active = tiles > 0;
     if (!active && bad_len && threadIdx.x == 0 && crank == 0) flag_status(p.status, OMNI_DEV_BAD_INDEX);
-    if (!active && !p.cluster_merge) c2_store_empty(p, b, s, h0, head_rows, warp, lane);
+    if (!kClusterMerge && !active) c2_store_empty(p, b, s, h0, head_rows, warp, lane);
 
     const uint32_t tmem = ctl->tmem_base;
     volatile uint32_t *abort_flag = &ctl->abort;
@@ -745,13 +748,13 @@ tc2q8_decode_kernel(const __grid_constant__ CUtensorMap q_nope_map, const __grid
             ok = mbar_wait(&ctl->x_bar, tiles & 1);
             ok = __all_sync(0xffffffffu, ok);
         }
-        if (ok && p.cluster_merge) {
+        if (kClusterMerge && ok) {
             if (warp == 2 && lane == 0) mbar_arrive_cluster(map_to_rank(smem_u32(&ctl->ready_bar), crank ^ 2u));
             const float lt = (ctl->xchg[tiles & 1][0][row] + ctl->xchg[tiles & 1][1][row]) +
                              (ctl->xchg[tiles & 1][2][row] + ctl->xchg[tiles & 1][3][row]);
             cm_inv = lt > 0.f ? 1.f / lt : 0.f;
             cm_lse = lt > 0.f ? (m_ref + log2f(lt)) * kLn2 : -INFINITY;
-        } else if (ok) {
+        } else if (!kClusterMerge && ok) {
             tc_fence_after();
             const float lt = (ctl->xchg[tiles & 1][0][row] + ctl->xchg[tiles & 1][1][row]) +
                              (ctl->xchg[tiles & 1][2][row] + ctl->xchg[tiles & 1][3][row]);
@@ -769,7 +772,7 @@ tc2q8_decode_kernel(const __grid_constant__ CUtensorMap q_nope_map, const __grid
     if (*abort_flag) {
         for (int i = 0; i < 200; ++i) __nanosleep(1000);
     }
-    if (p.cluster_merge) cluster_merge_exchange(p, ctl, smem, tmem, b, s, crank, h0, head_rows, active, softmax_ok, cm_lse, cm_inv);
+    if (kClusterMerge) cluster_merge_exchange(p, ctl, smem, tmem, b, s, crank, h0, head_rows, active, softmax_ok, cm_lse, cm_inv);
     tc_fence_before();
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -782,9 +785,25 @@ tc2q8_decode_kernel(const __grid_constant__ CUtensorMap q_nope_map, const __grid
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
-    if (p.cluster_merge) cluster_sync_relaxed();
-    if (p.splits > 1 && p.counters != nullptr)
+    if (kClusterMerge) cluster_sync_relaxed();
+    if (!kClusterMerge && p.splits > 1 && p.counters != nullptr)
         merge_if_last(p, b, (int)rank, 2, h0, head_rows, reinterpret_cast<float *>(smem), &ctl->merge_flag);
+}
+
+__global__ void __launch_bounds__(kC2Threads, 1)
+tc2q8_decode_kernel(const __grid_constant__ CUtensorMap q_nope_map, const __grid_constant__ CUtensorMap q_rope_map,
+                    const __grid_constant__ CUtensorMap kv_k_map, const __grid_constant__ CUtensorMap kv_v_map,
+                    const __grid_constant__ CUtensorMap kv_page_map, DecodeParams p)
+{
+    tc2q8_decode_body<false>(q_nope_map, q_rope_map, kv_k_map, kv_v_map, kv_page_map, p);
+}
+
+__global__ void __launch_bounds__(kC2Threads, 1)
+tc2q8_decode_cm_kernel(const __grid_constant__ CUtensorMap q_nope_map, const __grid_constant__ CUtensorMap q_rope_map,
+                       const __grid_constant__ CUtensorMap kv_k_map, const __grid_constant__ CUtensorMap kv_v_map,
+                       const __grid_constant__ CUtensorMap kv_page_map, DecodeParams p)
+{
+    tc2q8_decode_body<true>(q_nope_map, q_rope_map, kv_k_map, kv_v_map, kv_page_map, p);
 }
 
 // Quantiser of the 8-bit cache: one warp per row.  scale = max(amax, 2^-60) / 448 with amax the
@@ -847,7 +866,9 @@ inline bool tc2q8_prepare_device()
     std::lock_guard<std::mutex> lock(mu);
     if (!attr_set[dev]) {
         if (cudaFuncSetAttribute(tc2q8_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kC2SmemBytes) !=
-            cudaSuccess)
+                cudaSuccess ||
+            cudaFuncSetAttribute(tc2q8_decode_cm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kC2SmemBytes) !=
+                cudaSuccess)
             return false;
         attr_set[dev] = true;
     }
@@ -885,7 +906,8 @@ inline omni_status_t tc2q8_launch(const CUtensorMap *maps, const DecodeParams &p
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, tc2q8_decode_kernel, maps[0], maps[1], maps[2], maps[3], maps[4], p) == cudaSuccess
+    return cudaLaunchKernelEx(&cfg, p.cluster_merge ? tc2q8_decode_cm_kernel : tc2q8_decode_kernel, maps[0], maps[1], maps[2],
+                              maps[3], maps[4], p) == cudaSuccess
                ? OMNI_OK
                : OMNI_ERR_CUDA;
 }
