@@ -590,7 +590,8 @@ def main():
             "launch_bound": bool(host_us_per_call > 0.9 * ms_per_step * 1e3),
             "roofline": {"bound": "hbm", "achieved": round(achieved, 2), "peak": peaks["hbm"],
                          "unit": "GB/s", "frac": round(achieved / peaks["hbm"], 4),
-                         "traffic": _recorded_traffic(khash), "peak_source": peaks["source"],
+                         "traffic": (_recorded_traffic(khash) if args.workload == "config2" and args.batch == 32 else None),
+                         "peak_source": peaks["source"],
                          "kernel": "sparse_mla_decode main kernel (128 heads: tc2_decode_cm_kernel where two splits merge inside a cluster, as on the bench workload, else tc2_decode_kernel)", "kernel_us_mean": round(kmean * 1e3, 3),
                          "kernel_us_bracketed_min": round(min(kern_ms) * 1e3, 3),
                          "kernel_us_bracketed_mean": round(kbracket * 1e3, 3),
