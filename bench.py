@@ -522,9 +522,10 @@ def main():
                 torch.cuda.current_stream().wait_stream(ln["stream"])
 
     e2e_steps = args.steps
-    # the PCIe link needs a few milliseconds of traffic to leave its idle state, so this leg warms up
-    # with at least 100 steps whatever W is (untimed, like every warm-up step)
-    e2e_warmup = max(args.warmup, 100)
+    # the PCIe path needs some tens of milliseconds of traffic to reach its steady rate (the first few
+    # hundred steps after an idle period run 5 to 40 % slower), so this leg warms up with at least
+    # 500 steps whatever W is (untimed, like every warm-up step)
+    e2e_warmup = max(args.warmup, 500)
     fork_lanes()
     for i in range(e2e_warmup):
         e2e_step(i)
