@@ -161,6 +161,17 @@ __device__ __forceinline__ int64_t resolve_row(const int32_t *page_table_row, in
     return (int64_t)page * kPage + (t % kPage);
 }
 
+// 2^x for the softmax weights: the hardware approximation alone (ex2.approx.ftz, about 2 ulp,
+// -inf gives 0, results below 2^-126 are flushed to 0), where exp2f adds a range-scaling sequence
+// around it for subnormal results, four more instructions per weight in the hottest loop.  A
+// weight that small contributes nothing at the precision the weights are kept in.
+__device__ __forceinline__ float fast_exp2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 __device__ __forceinline__ void flag_status(int32_t *status, int32_t bits)
 {
     if (status != nullptr) atomicOr(status, bits);

@@ -1055,7 +1055,7 @@ __device__ __forceinline__ void tc2_decode_body(const CUtensorMap &q_map, const 
             uint32_t pk[16];
 #pragma unroll
             for (int j = 0; j < 32; j += 2) {
-                const float e0 = exp2f(x[j] - mr), e1 = exp2f(x[j + 1] - mr);
+                const float e0 = fast_exp2(x[j] - mr), e1 = fast_exp2(x[j + 1] - mr);
                 sum += e0 + e1;
                 pk[j >> 1] = pack_bf16(e0, e1);
             }

@@ -696,7 +696,7 @@ __device__ __forceinline__ void tc2q8_decode_body(const CUtensorMap &q_nope_map,
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     const int j = 4 * g + k;
-                    pw[j] = exp2f(y[j] - mr);                    // p * scale_t, below 448; 0 for a masked token
+                    pw[j] = fast_exp2(y[j] - mr);                    // p * scale_t, below 448; 0 for a masked token
                     sum += ((valid >> j) & 1u) ? pw[j] * rcv[k] : 0.f;      // p
                 }
             }
