@@ -1008,9 +1008,21 @@ __device__ __forceinline__ void tc2_decode_body(const CUtensorMap &q_map, const 
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(s_empty_leader + 8 * sbuf);
             const uint32_t valid = (uint32_t)(ctl->valid_mask[i % kMaskRing] >> (32 * half));
+            // x[j] * xs is the scaled score of token j.  A full tile under a positive scale keeps the
+            // raw scores (xs = the scale): the maximum is taken on them and the scale rides on the
+            // fused multiply-add in front of the exponential, one instruction less per token.
             float x[32];
             float mt = -INFINITY;
-            if (valid == 0xffffffffu) {
+            float xs = 1.f;
+            if (valid == 0xffffffffu && p.scale_log2 > 0.f) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    x[j] = __uint_as_float(sv[j]);
+                    mt = fmaxf(mt, x[j]);
+                }
+                xs = p.scale_log2;
+                mt *= xs;
+            } else if (valid == 0xffffffffu) {
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
                     x[j] = __uint_as_float(sv[j]) * p.scale_log2;
@@ -1055,7 +1067,7 @@ __device__ __forceinline__ void tc2_decode_body(const CUtensorMap &q_map, const 
             uint32_t pk[16];
 #pragma unroll
             for (int j = 0; j < 32; j += 2) {
-                const float e0 = fast_exp2(x[j] - mr), e1 = fast_exp2(x[j + 1] - mr);
+                const float e0 = fast_exp2(fmaf(x[j], xs, -mr)), e1 = fast_exp2(fmaf(x[j + 1], xs, -mr));
                 sum += e0 + e1;
                 pk[j >> 1] = pack_bf16(e0, e1);
             }
